@@ -244,3 +244,15 @@ def test_mixed_temperatures_and_ragged_offsets():
                                    T[b], [g], [0, g + 1], [0, g], gmax)
         assert one.n_accepted[0] == full.n_accepted[b]
         np.testing.assert_array_equal(one.out_tokens[0], full.out_tokens[b])
+
+
+def test_accept_comparison_is_strict():
+    # p uniform over 4 tokens (exactly 1/4), q a point mass on token 2 (exactly 1):
+    # ratio = 1/4 exactly; u = 1/4 is NOT below it -> reject; the next float32 below is accepted.
+    tl = np.zeros((2, 4), np.float32)
+    dl = np.array([[-np.inf, -np.inf, 0.0, -np.inf]], np.float32)
+    common = dict(temperature=1.0, gamma=[1], cu_q=[0, 2], cu_d=[0, 1], gamma_max=1)
+    r = oracle.accept_sample(tl, dl, [2], [0.25], [0.1], **common)
+    assert r.ratio[0] == 0.25 and r.n_accepted[0] == 0
+    r = oracle.accept_sample(tl, dl, [2], [np.nextafter(np.float32(0.25), np.float32(0))], [0.1], **common)
+    assert r.n_accepted[0] == 1
