@@ -1,0 +1,256 @@
+/*
+ * specverify -- the target model's verify step of speculative decoding with a
+ * draft length gamma that changes every step (GammaTune, "Token-Driven
+ * GammaTune: Adaptive Calibration for Enhanced Speculative Decoding").
+ *
+ * C ABI of a CUDA library for NVIDIA B200 (sm_100a).  Three operations make up
+ * one verify step; they run back to back on one stream and never synchronise
+ * with or read back to the host:
+ *
+ *   spec_verify_attn    attention of the gamma+1 draft positions against the
+ *                       paged bf16 KV cache                     (Section 3 / 5)
+ *   spec_accept_sample  accept / reject the drafts, resample or draw the bonus
+ *                       token                                   (Section 3)
+ *   gamma_tune_update   choose the next gamma from the number accepted
+ *                                                               (Section 4.1, Algorithm 1)
+ *
+ * General conventions
+ *   - Pointers named "device" point to device memory owned by the caller; the
+ *     library allocates no device memory and keeps no state between calls
+ *     except registered KV-pool handles (host memory).
+ *   - "host" pointers are plain host memory (spec_verify_step_host prefers
+ *     pinned memory so that its copies are asynchronous).
+ *   - Every call is asynchronous on the given stream (a cudaStream_t passed as
+ *     void*; NULL = the default stream) and returns after enqueueing.
+ *   - A negative sv_status is an error found on the host before anything was
+ *     launched.  Conditions found on the device (a page id outside the pool, a
+ *     token id outside the vocabulary, a non-finite softmax sum, gamma outside
+ *     [0, gamma_max], a bounded wait that expired) set bits in the caller's
+ *     device_status word; the affected sequence is skipped or clamped and the
+ *     kernel returns normally.  Nothing traps or asserts on the device.
+ *   - Batch notation: B sequences; sequence b has draft length gamma[b] and
+ *     R_b = gamma[b]+1 query / target rows starting at row cu_q[b], and
+ *     gamma[b] draft rows / tokens / uniforms starting at cu_d[b].  seq_len[b]
+ *     is the KV length INCLUDING those R_b positions (their K/V are already in
+ *     the cache).  gamma, seq_len, cu_q, cu_d live on the device.
+ */
+#ifndef SPECVERIFY_H
+#define SPECVERIFY_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t sv_status;
+enum {
+    SV_OK = 0,
+    SV_EINVAL = -1,        /* null pointer, non-positive size, inconsistent arguments */
+    SV_EUNSUPPORTED = -2,  /* head_dim not 64/128, page_size not 16, hq % hkv != 0, ... */
+    SV_EALIGN = -3,        /* a pointer or stride misses the alignment stated below */
+    SV_ECUDA = -4,         /* a CUDA runtime / driver call failed (launch, tensor map) */
+    SV_EWORKSPACE = -5     /* workspace missing or smaller than the size query says */
+};
+
+/* bits of the device status word */
+enum {
+    SV_DEV_BAD_GAMMA = 1,   /* gamma[b] outside [0, gamma_max]: clamped */
+    SV_DEV_BAD_PAGE = 2,    /* block-table entry outside [0, n_pages): sequence skipped */
+    SV_DEV_BAD_TOKEN = 4,   /* draft token outside [0, vocab): position rejected */
+    SV_DEV_NONFINITE = 8,   /* softmax sum not finite (NaN / +Inf logit): sequence emits -1 */
+    SV_DEV_TIMEOUT = 16,    /* a bounded device-side wait expired */
+    SV_DEV_BAD_LEN = 32     /* seq_len[b] < gamma[b]+1 or beyond the block table: sequence skipped */
+};
+
+const char *sv_status_str(sv_status s);
+
+/* ---------------------------------------------------------------- KV pool */
+/*
+ * A paged KV pool: K and V arrays of n_pages pages, each page holding
+ * page_size (= 16) token slots for hkv heads of head_dim bf16 values.
+ * strides[4] = element strides for (page, kv head, slot, dim); dim stride must
+ * be 1, the others multiples of 8 elements (16 bytes); both base pointers
+ * 16-byte aligned.  [page, head, slot, dim] and [page, slot, head, dim] are
+ * both expressible.  Registration builds the TMA tensor maps on the host; the
+ * handle is host memory released by spec_kv_pool_release.  Slots past a
+ * sequence's seq_len inside its last page are read (and multiplied by zero
+ * weights), so pool memory must hold finite values.
+ */
+typedef struct sv_kv_pool *sv_kv_pool_t;
+
+sv_status spec_kv_pool_register(const void *k_pool_device, const void *v_pool_device,
+                                int64_t n_pages, int32_t page_size, int32_t hkv, int32_t head_dim,
+                                const int64_t strides[4], sv_kv_pool_t *out);
+sv_status spec_kv_pool_release(sv_kv_pool_t pool);
+
+/* ---------------------------------------------------------------- attention */
+/*
+ * Paper Section 3: the target verifies the gamma drafted tokens in one parallel
+ * forward; with KV caching (Section 5) the context-dependent part of it is
+ * this causal attention.  For sequence b, row i in [0, gamma[b]], query head h:
+ *     pos = seq_len[b] - (gamma[b]+1) + i ;  kv head = h / (hq / hkv)
+ *     s_j = sm_scale * <q, k_j>   for j = 0 .. pos
+ *     o   = sum_j softmax(s)_j v_j ;   lse = ln sum_j exp(s_j)
+ * bf16 inputs, fp32 accumulation and softmax, bf16 output.
+ */
+typedef struct sv_attn_params {
+    const void *q;              /* device bf16 [n_rows, hq, head_dim], 16-byte aligned */
+    void *o;                    /* device bf16 [n_rows, hq, head_dim], 16-byte aligned */
+    float *lse;                 /* device fp32 [n_rows, hq], or NULL */
+    sv_kv_pool_t pool;
+    const int32_t *block_table; /* device [batch, block_table_stride]: physical page of logical page */
+    int64_t block_table_stride; /* elements between rows; >= ceil(max_seq_len / 16) */
+    const int32_t *seq_len;     /* device [batch] */
+    const int32_t *gamma;       /* device [batch] */
+    const int32_t *cu_q;        /* device [batch+1] */
+    int32_t batch;
+    int32_t gamma_max;          /* upper bound of gamma[b]; sizes the row tile */
+    int32_t hq, hkv, head_dim;
+    int32_t max_seq_len;        /* upper bound of seq_len[b]; sizes the grid and the workspace */
+    float sm_scale;             /* usually 1/sqrt(head_dim) */
+    uint32_t *device_status;    /* device, one word, OR-ed into; may be NULL */
+} sv_attn_params;
+
+/* Bytes of device scratch spec_verify_attn needs for these bounds (partial
+ * results of sequences whose keys are split over several thread blocks). */
+size_t spec_verify_attn_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t hq, int32_t hkv,
+                                        int32_t head_dim, int32_t max_seq_len);
+
+sv_status spec_verify_attn(const sv_attn_params *p, void *workspace_device, size_t workspace_bytes,
+                           void *stream);
+
+/* ---------------------------------------------------------------- accept / resample */
+/*
+ * Speculative sampling (paper Section 3, after Leviathan et al. and Chen et
+ * al.).  Per sequence, with T = its temperature, target rows t_0..t_gamma and
+ * draft rows d_0..d_{gamma-1}, draft tokens x_i, uniforms u_i and u_s:
+ *   T > 0:  p_i = softmax(t_i / T), q_i = softmax(d_i / T)
+ *           ratio_i = min(1, p_i[x_i] / q_i[x_i]); accept while u_i < ratio_i;
+ *           n = index of the first rejection (gamma if none)
+ *           n < gamma: next ~ normalise(max(0, p_n - q_n))  (p_n if that is all zero)
+ *           n = gamma: next ~ p_gamma                        (the bonus token)
+ *           both by inverse CDF in vocabulary order with u_s
+ *           (smallest k with sum_{j<=k} w_j > u_s * sum_j w_j).
+ *   T == 0: n = first i with argmax(t_i) != x_i (lowest index wins ties),
+ *           next = argmax(t_n); draft logits and uniforms are not read.
+ * Softmax sums are accumulated in float64 from float32 exponentials; the
+ * ratio, the comparison and the sampled row are evaluated in float64.
+ */
+typedef struct sv_accept_params {
+    const float *target_logits;   /* device fp32 [n_q_rows, row_stride] */
+    const float *draft_logits;    /* device fp32 [n_d_rows, row_stride]; may be NULL if all T == 0 */
+    int64_t row_stride;           /* elements between rows (>= vocab); a multiple of 4 with
+                                     16-byte aligned bases enables 128-bit loads */
+    int32_t vocab;
+    const int32_t *draft_tokens;  /* device [n_d_rows] */
+    const float *u_accept;        /* device [n_d_rows], in [0,1) */
+    const float *u_sample;        /* device [batch], in [0,1) */
+    float temperature;            /* used when temperature_per_seq is NULL */
+    const float *temperature_per_seq; /* device [batch] or NULL */
+    const int32_t *gamma;         /* device [batch] */
+    const int32_t *cu_q;          /* device [batch+1] */
+    const int32_t *cu_d;          /* device [batch+1] */
+    int32_t batch;
+    int32_t gamma_max;
+    int32_t *n_accepted;          /* device out [batch]: accepted drafts, 0..gamma (extra token not counted) */
+    int32_t *out_tokens;          /* device out [batch, gamma_max+1]: accepted drafts, next token, then -1 */
+    double *ratio;                /* device out [n_d_rows] or NULL (NaN past the first rejection) */
+    double *logZ_p;               /* device out [n_q_rows] or NULL: ln sum exp(t/T) */
+    double *logZ_q;               /* device out [n_d_rows] or NULL: ln sum exp(d/T) */
+    uint32_t *flag_count;         /* device, one word or NULL: += positions with |u - ratio| < 1e-6 */
+    uint32_t *device_status;      /* device, one word or NULL */
+} sv_accept_params;
+
+size_t spec_accept_sample_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t vocab);
+
+sv_status spec_accept_sample(const sv_accept_params *p, void *workspace_device,
+                             size_t workspace_bytes, void *stream);
+
+/* ---------------------------------------------------------------- GammaTune */
+/*
+ * Paper Section 4.1, Algorithm 1, one update per sequence, state on the device:
+ *   SV_GT_PROPOSED  A' = A + delta if A == gamma else A      (Eq. 7 feeding the average,
+ *                   gbar <- min(gmax, max(gmin, (1-eta) gbar + eta A'))   (Eq. 8)   as the prose says)
+ *                   gamma <- ceil(gbar)
+ *   SV_GT_LITERAL   the listing as printed: the average is fed A itself
+ *   SV_GT_FIXED     gamma and gbar stay (plain speculative decoding)
+ * binary64 throughout, each product and the sum rounded separately (no fused
+ * multiply-add), so trajectories are reproducible bit for bit.
+ * Bookkeeping done in the same kernel:
+ *   seq_len <- seq_len - (gamma+1) + (A+1) + (gamma_next+1)
+ *   cu_q, cu_d <- prefix sums of gamma_next+1 / gamma_next, or b*(gamma_max+1) /
+ *   b*gamma_max when padded_rows != 0 (fixed row slabs per sequence).
+ */
+enum { SV_GT_FIXED = 0, SV_GT_PROPOSED = 1, SV_GT_LITERAL = 2 };
+
+typedef struct sv_gamma_config {
+    double eta;          /* adaptation rate in [0, 1] */
+    double delta;        /* expansion offset */
+    int32_t gamma_min;   /* >= 0 */
+    int32_t gamma_max;   /* >= gamma_min */
+    int32_t mode;        /* SV_GT_* */
+    int32_t padded_rows; /* row-offset convention, see above */
+} sv_gamma_config;
+
+typedef struct sv_gamma_params {
+    const int32_t *n_accepted;  /* device [batch] */
+    double *gamma_bar;          /* device in/out [batch] */
+    int32_t *gamma;             /* device in/out [batch] */
+    int32_t *seq_len;           /* device in/out [batch], or NULL */
+    int32_t *cu_q;              /* device out [batch+1] */
+    int32_t *cu_d;              /* device out [batch+1] */
+    int32_t batch;
+    sv_gamma_config config;
+    int32_t *trajectory;        /* device out or NULL: gamma_next written to trajectory[step*batch + b] */
+    int32_t *accepted_log;      /* device out or NULL: A written to accepted_log[step*batch + b] */
+    int32_t step;
+    uint32_t *device_status;    /* device, one word or NULL */
+} sv_gamma_params;
+
+sv_status gamma_tune_update(const sv_gamma_params *p, void *stream);
+/* gamma = gamma0 and gamma_bar = gamma0 for every sequence, cu_q / cu_d built; n_accepted,
+ * seq_len, trajectory are not touched. */
+sv_status gamma_tune_init(const sv_gamma_params *p, int32_t gamma0, void *stream);
+
+/* ---------------------------------------------------------------- whole step from host buffers */
+/*
+ * One verify step whose per-step inputs start in HOST memory: copies q,
+ * logits, draft tokens and uniforms to the caller's device staging buffers,
+ * runs spec_verify_attn, spec_accept_sample, gamma_tune_update on `stream`,
+ * and copies n_accepted, out_tokens, gamma (next) and the attention output
+ * back to host buffers.  All asynchronous; the caller synchronises the stream
+ * before reading the host outputs.  The KV pool, block table and controller
+ * state stay resident on the device (that is what a KV cache is).
+ * n_q_rows / n_d_rows are the numbers of rows to copy (host knows the layout
+ * it filled).  Device pointers inside attn / accept / gamma are used as the
+ * staging destinations.
+ */
+typedef struct sv_step_host_io {
+    const void *q_host;             /* bf16 [n_q_rows, hq, head_dim] */
+    const float *target_logits_host;
+    const float *draft_logits_host;
+    const int32_t *draft_tokens_host;
+    const float *u_accept_host;
+    const float *u_sample_host;
+    int64_t n_q_rows, n_d_rows;
+    int32_t *n_accepted_host;       /* out [batch] */
+    int32_t *out_tokens_host;       /* out [batch, gamma_max+1] */
+    int32_t *gamma_next_host;       /* out [batch] */
+    void *o_host;                   /* out bf16 [n_q_rows, hq, head_dim], or NULL */
+} sv_step_host_io;
+
+sv_status spec_verify_step_host(const sv_step_host_io *io, const sv_attn_params *attn,
+                                void *attn_workspace, size_t attn_workspace_bytes,
+                                const sv_accept_params *accept, void *accept_workspace,
+                                size_t accept_workspace_bytes, const sv_gamma_params *gamma,
+                                void *stream);
+
+/* Kernel launches issued by the library since it was loaded (for reporting). */
+uint64_t sv_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECVERIFY_H */

@@ -142,8 +142,8 @@ def accept_sample(target_logits, draft_logits, draft_tokens, u_accept, u_sample,
     n_d, n_q = int(cd[B]), int(cq[B])
     res = AcceptResult(
         n_accepted=np.zeros(B, np.int32), out_tokens=np.zeros((B, gamma_max + 1), np.int32),
-        ratio=np.zeros(max(n_d, 1), np.float64), logZ_p=np.zeros(max(n_q, 1), np.float64),
-        logZ_q=np.zeros(max(n_d, 1), np.float64), accept_flag=np.zeros(max(n_d, 1), np.uint8),
+        ratio=np.full(max(n_d, 1), np.nan), logZ_p=np.full(max(n_q, 1), np.nan),
+        logZ_q=np.full(max(n_d, 1), np.nan), accept_flag=np.zeros(max(n_d, 1), np.uint8),
         alt_token=np.zeros(B, np.int32), sample_flag=np.zeros(B, np.uint8),
         resid_mass=np.zeros(B, np.float64))
     fptr = None
