@@ -168,6 +168,38 @@ size_t spec_accept_sample_workspace_bytes(int32_t batch, int32_t gamma_max, int3
 sv_status spec_accept_sample(const sv_accept_params *p, void *workspace_device,
                              size_t workspace_bytes, void *stream);
 
+/*
+ * spec_accept_sample without a workspace argument and without any allocation.
+ * The paper has no counterpart to this entry point; it exists for callers that
+ * are not able to obtain device scratch memory themselves: code running where
+ * every device buffer was fixed at start-up (a serving engine whose memory pool
+ * is fully handed out, a plugin that is only given its input and output
+ * tensors), or code that must not call cudaMalloc at this point because an
+ * allocation would synchronise the device or is forbidden by the host
+ * framework's rules.  The computation and the results are those of
+ * spec_accept_sample; only the place of the intermediate slice statistics
+ * differs: they go to an array of SV_ACCEPT_STATIC_SCRATCH_BYTES bytes that is
+ * built into the library (each GPU that loads the library carries it until the
+ * process ends).
+ *   - Limit: batch * (2*gamma_max + 1) * slices * 32 bytes must not exceed
+ *     SV_ACCEPT_STATIC_SCRATCH_BYTES, where slices = ceil(vocab / slice) and the
+ *     library picks slice between 2048 and 16384 elements (larger when there are
+ *     many rows).  The largest configuration of the tests (batch 128, gamma_max
+ *     16, vocab 128256) needs about 1.1 MB.  A larger problem is refused with
+ *     SV_EWORKSPACE before anything is launched; use spec_accept_sample then.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress) with that device current; make that first call
+ *     outside any stream capture.  No call allocates or frees memory.
+ *   - All calls on one device share the array and it keeps whatever the previous
+ *     call left there.  Nothing needs clearing: every record a call reads was
+ *     written earlier in that same call.  Two calls whose kernels can overlap on
+ *     the GPU (different streams without an ordering between them) race on the
+ *     array and give wrong results; keep such calls on one stream or order them
+ *     with events.
+ */
+#define SV_ACCEPT_STATIC_SCRATCH_BYTES (4u << 20)
+sv_status spec_accept_sample_static(const sv_accept_params *p, void *stream);
+
 /* ---------------------------------------------------------------- GammaTune */
 /*
  * Paper Section 4.1, Algorithm 1, one update per sequence, state on the device:

@@ -24,7 +24,8 @@ SV_GT_FIXED, SV_GT_PROPOSED, SV_GT_LITERAL = 0, 1, 2
 EXPORTS = (
     "sv_status_str", "sv_launch_count", "spec_kv_pool_register", "spec_kv_pool_release",
     "spec_verify_attn_workspace_bytes", "spec_verify_attn", "spec_accept_sample_workspace_bytes",
-    "spec_accept_sample", "gamma_tune_update", "gamma_tune_init", "spec_verify_step_host",
+    "spec_accept_sample", "spec_accept_sample_static", "gamma_tune_update", "gamma_tune_init",
+    "spec_verify_step_host",
 )
 
 
@@ -103,6 +104,8 @@ def load():
         lib.spec_verify_attn.argtypes = [C.POINTER(AttnParams), C.c_void_p, C.c_size_t, C.c_void_p]
         lib.spec_accept_sample.restype = C.c_int32
         lib.spec_accept_sample.argtypes = [C.POINTER(AcceptParams), C.c_void_p, C.c_size_t, C.c_void_p]
+        lib.spec_accept_sample_static.restype = C.c_int32
+        lib.spec_accept_sample_static.argtypes = [C.POINTER(AcceptParams), C.c_void_p]
         lib.gamma_tune_update.restype = C.c_int32
         lib.gamma_tune_update.argtypes = [C.POINTER(GammaParams), C.c_void_p]
         lib.gamma_tune_init.restype = C.c_int32
@@ -285,6 +288,22 @@ def spec_accept_sample(target_logits, draft_logits, draft_tokens, u_accept, u_sa
     _check("spec_accept_sample",
            load().spec_accept_sample(C.byref(p), workspace.data_ptr(), _nbytes(workspace),
                                      _stream(stream)))
+
+
+SV_ACCEPT_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def spec_accept_sample_static(target_logits, draft_logits, draft_tokens, u_accept, u_sample, temperature,
+                              gamma, cu_q, cu_d, gamma_max, n_accepted, out_tokens, ratio=None,
+                              logZ_p=None, logZ_q=None, flag_count=None, device_status=None,
+                              temperature_per_seq=None, stream=None):
+    """spec_accept_sample for callers that cannot hand over scratch memory (no workspace
+    argument; the library's built-in array is used).  Problems beyond that array's size raise
+    SpecVerifyError with SV_EWORKSPACE.  Calls on one device must not overlap on the GPU."""
+    p = accept_params(target_logits, draft_logits, draft_tokens, u_accept, u_sample, temperature,
+                      gamma, cu_q, cu_d, gamma_max, n_accepted, out_tokens, ratio, logZ_p, logZ_q,
+                      flag_count, device_status, temperature_per_seq)
+    _check("spec_accept_sample_static", load().spec_accept_sample_static(C.byref(p), _stream(stream)))
 
 
 # --------------------------------------------------------------------------- GammaTune

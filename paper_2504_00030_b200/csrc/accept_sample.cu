@@ -573,3 +573,73 @@ extern "C" sv_status spec_accept_sample(const sv_accept_params *p, void *workspa
     sv::accept_finish_kernel<<<p->batch, sv::FIN_THREADS, dyn, (cudaStream_t)stream>>>(a);
     return sv::launch_check();
 }
+
+// ---------------------------------------------------------------------------------------------
+// Variant without caller-provided scratch.
+// ---------------------------------------------------------------------------------------------
+namespace sv {
+
+// Slice statistics of one call live here instead of in a caller's workspace.  The array is part
+// of the library image: every GPU that loads the library holds these bytes until the process
+// exits.  All calls on a device share it.
+static __device__ __align__(256) unsigned char g_accept_static_scratch[SV_ACCEPT_STATIC_SCRATCH_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+static void *g_static_scratch_ptr[MAX_DEVICES];   // device address of the array, per device
+
+}  // namespace sv
+
+extern "C" sv_status spec_accept_sample_static(const sv_accept_params *p, void *stream)
+{
+    if (p == nullptr || p->batch <= 0 || p->vocab <= 0 || p->gamma_max < 0) return SV_EINVAL;
+    if (p->gamma_max > 64) return SV_EUNSUPPORTED;
+    if (p->target_logits == nullptr || p->gamma == nullptr || p->cu_q == nullptr ||
+        p->cu_d == nullptr || p->n_accepted == nullptr || p->out_tokens == nullptr)
+        return SV_EINVAL;
+    const bool any_sampling = p->temperature_per_seq != nullptr || p->temperature > 0.f;
+    if (any_sampling && (p->draft_logits == nullptr || p->u_accept == nullptr || p->u_sample == nullptr))
+        return SV_EINVAL;
+    if (p->gamma_max > 0 && p->draft_tokens == nullptr) return SV_EINVAL;
+    if (p->row_stride < p->vocab) return SV_EINVAL;
+    if (!(p->temperature >= 0.f)) return SV_EINVAL;
+    const int n_seg = (p->vocab + sv::SEG - 1) / sv::SEG;
+    const size_t dyn = 3 * sizeof(double) * (size_t)n_seg;
+    if (dyn > 200 * 1024) return SV_EUNSUPPORTED;
+
+    sv::AcceptLaunch a;
+    a.p = *p;
+    a.slice = sv::pick_slice(p);
+    a.n_slices = (p->vocab + a.slice - 1) / a.slice;
+    a.vec_ok = (p->row_stride % 4 == 0) && sv::aligned16(p->target_logits) &&
+               (p->draft_logits == nullptr || sv::aligned16(p->draft_logits));
+    const unsigned long long n_items =
+        (unsigned long long)p->batch * (2ull * p->gamma_max + 1) * (unsigned long long)a.n_slices;
+    // the problem must fit the built-in array: one 32-byte record per (row, slice)
+    if (n_items * sizeof(sv::RowPartial) > (unsigned long long)SV_ACCEPT_STATIC_SCRATCH_BYTES)
+        return SV_EWORKSPACE;
+
+    // In host code the array's name is only a handle; its device address has to be asked for,
+    // once per device, with that device current.
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= sv::MAX_DEVICES) return SV_ECUDA;
+    if (sv::g_static_scratch_ptr[dev] == nullptr) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, sv::g_accept_static_scratch) != cudaSuccess || ptr == nullptr)
+            return SV_ECUDA;
+        sv::g_static_scratch_ptr[dev] = ptr;
+    }
+    a.partials = static_cast<sv::RowPartial *>(sv::g_static_scratch_ptr[dev]);
+
+    const long long cap = 8LL * sv::sm_count();
+    const int grid = (int)((long long)n_items < cap ? (long long)n_items : cap);
+    sv::accept_rowstats_kernel<<<grid, sv::RS_THREADS, 0, (cudaStream_t)stream>>>(a);
+    sv_status st = sv::launch_check();
+    if (st != SV_OK) return st;
+    if (dyn > 48 * 1024) {
+        if (cudaFuncSetAttribute(sv::accept_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)dyn) != cudaSuccess)
+            return SV_ECUDA;
+    }
+    sv::accept_finish_kernel<<<p->batch, sv::FIN_THREADS, dyn, (cudaStream_t)stream>>>(a);
+    return sv::launch_check();
+}
