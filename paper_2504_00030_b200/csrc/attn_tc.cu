@@ -1,7 +1,777 @@
-// placeholder until the tensor-core kernel lands
+// Draft-block attention on the 5th-generation tensor cores (tcgen05, sm_100a).
+//
+// Work unit.  A (sequence b, kv head g) pair owns G*(gamma_b+1) query rows (G = hq/hkv query
+// heads per kv head, stacked so that the group shares one pass over the keys) and a stream of
+// ceil(L_b/128) key tiles of 128 tokens = 8 pages.  The key tiles of the whole batch form one
+// global list; each of the grid's persistent thread blocks takes an equal contiguous share of
+// it (lengths live on the device, so the split is computed in the kernel), which balances ragged
+// contexts exactly.  A block's share is cut into segments, one per (b, g) it touches; a segment
+// that covers its pair completely writes the final output, otherwise it leaves an unnormalised
+// partial (fp32 O, running max, running sum) in the workspace for attn_combine_kernel.
+//
+// Data path per tile: the 8 K pages and 8 V pages are fetched by TMA (one 4-D tensor map over
+// the pool, box = 64 dims x 16 slots of one head of one page, 128-byte swizzle) into a ring of
+// 32 KB shared-memory slots, straight into the layout tcgen05 wants.  S = Q K^T is issued as
+// 8 MMAs (M=128 rows, N=128 tokens, K=16) with both operands in shared memory and the
+// accumulator in tensor memory; 128 softmax threads (one per query row, the row's scores in
+// their own TMEM lane, so max and sum need no shuffles) turn S into bf16 P in place; O += P V
+// is 8 MMAs with P read from tensor memory and V (token-major in memory) as the N-major B
+// operand.  Rows beyond 128 (e.g. 8 heads x 17 positions = 136) go to a second row group with
+// its own S / O accumulators and softmax warps; the two groups alternate on the tensor core.
+//
+// Warps: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 4..7 = softmax / epilogue of row
+// group 0, 8..11 = row group 1 (when needed).  All hand-offs are mbarriers; every wait is
+// bounded and an expired wait sets SV_DEV_TIMEOUT and drains the block.
 #include "attn_common.cuh"
+
+#include <math_constants.h>
+
 namespace sv {
-bool attn_tc_supported(const sv_attn_params &) { return false; }
-size_t attn_tc_workspace_bytes(int32_t, int32_t, int32_t, int32_t, int32_t, int32_t) { return 0; }
-sv_status launch_attn_tc(const sv_attn_params &, void *, size_t, cudaStream_t) { return SV_EUNSUPPORTED; }
+
+constexpr int TILE = 128;               // tokens per tile
+constexpr int PAGES_PER_TILE = 8;
+constexpr int HD = 128;                 // head_dim of this kernel
+constexpr int SLOT_BYTES = TILE * HD * 2;          // 32 KB: one K or one V tile
+constexpr int QGROUP_BYTES = 128 * HD * 2;         // 32 KB: 128 query rows
+constexpr int MAX_BATCH_TC = 1 << 20;
+constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2 s: far beyond any legitimate wait
+constexpr float RESCALE_THRESHOLD = 8.f;           // log2 units: P <= 2^8 before a lazy rescale
+
+// ---------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        " selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, int c0, int c1,
+                                            int c2, int c3, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.u32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.u32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(d),
+        "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+          "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+          "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+          "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
+        "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
+        "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  Tiles are stored as two 16 KB halves
+// (64 of the 128 dims each), each half as rows of 128 bytes (one token or one query row),
+// groups of 8 rows = 1024 bytes.
+//   K-major (Q as A, K as B): stride between 8-row groups = 1024; leading offset unused.
+//   N-major (V as B, N = dim): the 8 K-rows (tokens) of a group are 128 bytes apart, groups
+//   1024 bytes apart (stride offset), the second 64 dims 16 KB further (leading offset).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;      // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;      // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128.
+__device__ __forceinline__ uint32_t instr_desc(bool b_n_major)
+{
+    uint32_t d = 0;
+    d |= 1u << 4;                 // accumulator fp32
+    d |= 1u << 7;                 // A bf16
+    d |= 1u << 10;                // B bf16
+    d |= (b_n_major ? 1u : 0u) << 16;
+    d |= (uint32_t)(128 >> 3) << 17;
+    d |= (uint32_t)(128 >> 4) << 24;
+    return d;
+}
+
+// ---------------------------------------------------------------------------- schedule
+struct AttnTcLaunch {
+    sv_attn_params p;
+    int64_t n_pool_pages;
+    int group;           // query heads per kv head
+    int nq;              // row groups of 128 rows (1 or 2)
+    int n_slots;         // K/V ring slots
+    int32_t *ws_prefix;  // [batch+1] tile prefix, then [2]: total tiles, grid size
+    float *ws_part;      // partial results: slot-major
+};
+
+__host__ __device__ inline size_t part_slot_floats(int nq) { return (size_t)nq * 128 * (HD + 2); }
+
+// first global tile of block c when `total` tiles are split over `grid` blocks
+__device__ __forceinline__ long long share_begin(long long c, long long total, long long grid)
+{
+    return (c * total) / grid;
+}
+
+struct Shared {
+    uint64_t full[8];        // ring slot filled by TMA
+    uint64_t empty[8];       // ring slot released by the tensor core
+    uint64_t s_full[2];      // S accumulator ready
+    uint64_t p_full[2];      // P written by the softmax threads
+    uint64_t o_done[2];      // PV of a row group finished
+    uint64_t q_full;         // query rows of a segment are in shared memory
+    uint32_t tmem_base;
+    int abort_flag;
+    int total_tiles;         // sum over sequences of ceil(L/128)
+    int start_b;             // sequence that holds this block's first tile
+    int start_prefix;        // tiles (per kv head) of the sequences before it
+};
+
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, Shared *sh, uint32_t *status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int it = 0; it < 256; ++it)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*(volatile int *)&sh->abort_flag) return false;
+        if (clock64() - t0 > WAIT_CYCLES) break;
+    }
+    *(volatile int *)&sh->abort_flag = 1;
+    set_status(status, SV_DEV_TIMEOUT);
+    return false;
+}
+
+// Tiles and validated gamma of one sequence; sequences with inconsistent lengths own no tiles.
+__device__ __forceinline__ int seq_tiles(const sv_attn_params &p, int b, int *gam_out, bool report)
+{
+    int g = p.gamma[b];
+    if (g < 0 || g > p.gamma_max) {
+        if (report) set_status(p.device_status, SV_DEV_BAD_GAMMA);
+        g = min(max(g, 0), p.gamma_max);
+    }
+    const int L = p.seq_len[b];
+    int nt = (L + TILE - 1) / TILE;
+    if (L < g + 1 || (long long)(L + 15) / 16 > p.block_table_stride || L > p.max_seq_len) {
+        if (report) set_status(p.device_status, SV_DEV_BAD_LEN);
+        nt = 0;
+    }
+    if (gam_out != nullptr) *gam_out = g;
+    return nt;
+}
+
+// Walks the (sequence, kv head, tile) triples of a block's share.
+struct TileCursor {
+    int b, g, t, n_tiles, gam;    // current pair, tile inside it, its tile count and gamma
+    __device__ void seek(const sv_attn_params &p, const Shared *sh, long long tile)
+    {
+        b = sh->start_b;
+        n_tiles = seq_tiles(p, b, &gam, false);
+        const long long rel = tile - (long long)sh->start_prefix * p.hkv;
+        g = (int)(rel / n_tiles);
+        t = (int)(rel % n_tiles);
+    }
+    __device__ void next_pair(const sv_attn_params &p)
+    {
+        t = 0;
+        if (++g == p.hkv) {
+            g = 0;
+            n_tiles = 0;
+            while (n_tiles == 0 && ++b < p.batch) n_tiles = seq_tiles(p, b, &gam, false);
+            if (b >= p.batch) n_tiles = 1;      // past the end: never used
+        }
+    }
+};
+
+// ---------------------------------------------------------------------------- main kernel
+template <int NQ>
+__global__ void __launch_bounds__(128 + 128 * NQ, 1)
+attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
+               const __grid_constant__ CUtensorMap v_map)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    // carve: [Q groups][ring slots][Shared]; the dynamic window is aligned to 1024 by the launch
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *q_smem = smem;
+    uint8_t *ring = smem + NQ * QGROUP_BYTES;
+    Shared *sh = reinterpret_cast<Shared *>(ring + a.n_slots * SLOT_BYTES);
+
+    const sv_attn_params &p = a.p;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int batch = p.batch, hkv = p.hkv, G = a.group;
+    const int n_slots = a.n_slots;
+
+    // ---- tile prefix over the batch (every block computes the same thing)
+    if (tid == 0) {
+        for (int i = 0; i < n_slots; ++i) {
+            mbar_init(smem_u32(&sh->full[i]), 1);
+            mbar_init(smem_u32(&sh->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&sh->s_full[i]), 1);
+            mbar_init(smem_u32(&sh->p_full[i]), 128);
+            mbar_init(smem_u32(&sh->o_done[i]), 1);
+        }
+        mbar_init(smem_u32(&sh->q_full), 128 * NQ);
+        sh->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 0) {
+        // pass 1: total tiles; block 0 also publishes the inclusive prefix for the combine kernel
+        int carry = 0;
+        if (blockIdx.x == 0 && lane == 0) a.ws_prefix[0] = 0;
+        for (int base = 0; base < batch; base += 32) {
+            const int b = base + lane;
+            int v = (b < batch) ? seq_tiles(p, b, nullptr, blockIdx.x == 0) : 0;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, v, d);
+                if (lane >= d) v += t;
+            }
+            if (blockIdx.x == 0 && b < batch) a.ws_prefix[b + 1] = carry + v;
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+        const long long total = (long long)carry * hkv;
+        const long long my_begin = share_begin(blockIdx.x, total, gridDim.x);
+        if (lane == 0) {
+            sh->total_tiles = carry;
+            sh->start_b = 0;
+            sh->start_prefix = 0;
+            if (blockIdx.x == 0) a.ws_prefix[batch + 1] = (int)gridDim.x;
+        }
+        __syncwarp();
+        // pass 2: the sequence whose tiles contain this block's first tile
+        carry = 0;
+        for (int base = 0; base < batch; base += 32) {
+            const int b = base + lane;
+            const int nt = (b < batch) ? seq_tiles(p, b, nullptr, false) : 0;
+            int v = nt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, v, d);
+                if (lane >= d) v += t;
+            }
+            const long long lo = (long long)(carry + v - nt) * hkv, hi = (long long)(carry + v) * hkv;
+            if (nt > 0 && lo <= my_begin && my_begin < hi) {
+                sh->start_b = b;
+                sh->start_prefix = carry + v - nt;
+            }
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(&sh->tmem_base)),
+                     "r"(512u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    const long long total = (long long)sh->total_tiles * hkv;
+    const long long grid = gridDim.x;
+    const long long t_begin = share_begin(blockIdx.x, total, grid);
+    const long long t_end = share_begin(blockIdx.x + 1, total, grid);
+    const uint32_t tmem = sh->tmem_base;
+    const float c_scale = p.sm_scale * 1.4426950408889634f;   // scores in log2 units
+
+    if (t_end > t_begin) {
+        if (warp == 0) {
+            // ================================================================ TMA producer
+            TileCursor cur;
+            cur.seek(p, sh, t_begin);
+            uint32_t item = 0;     // ring items: 2*tile = K, 2*tile+1 = V
+            for (long long tg = t_begin; tg < t_end; ++tg) {
+                const int b = cur.b;
+                const int L = p.seq_len[b];
+                const int n_pages = (L + 15) >> 4;
+                const int32_t *bt = p.block_table + (long long)b * p.block_table_stride;
+                // lane l fetches (page l/2, dims half l%2) of K, then of V
+                const int page_in_tile = (lane & 15) >> 1, half = lane & 1;
+                const int lp = cur.t * PAGES_PER_TILE + page_in_tile;
+                int phys = (int)a.n_pool_pages;       // out of range: TMA fills zeros, no traffic
+                if (lp < n_pages) {
+                    const int e = bt[lp];
+                    if (e < 0 || e >= a.n_pool_pages) set_status(p.device_status, SV_DEV_BAD_PAGE);
+                    else phys = e;
+                }
+                bool ok = true;
+#pragma unroll
+                for (int kv = 0; kv < 2; ++kv) {
+                    const uint32_t slot = item % (uint32_t)n_slots;
+                    const uint32_t use = item / (uint32_t)n_slots;
+                    const uint32_t full = smem_u32(&sh->full[slot]);
+                    if (use > 0) ok = ok && bounded_wait(smem_u32(&sh->empty[slot]), (use - 1) & 1, sh, p.device_status);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    if (lane == 0) mbar_expect_tx(full, SLOT_BYTES);
+                    __syncwarp();
+                    if (lane < 16) {
+                        const uint32_t dst = smem_u32(ring + slot * SLOT_BYTES + half * (SLOT_BYTES / 2) +
+                                                      page_in_tile * 2048);
+                        tma_load_4d(dst, kv == 0 ? &k_map : &v_map, half * 64, 0, cur.g, phys, full);
+                    }
+                    ++item;
+                }
+                if (!ok) break;
+                if (++cur.t == cur.n_tiles) cur.next_pair(p);
+            }
+        } else if (warp == 1) {
+            // ================================================================ MMA issuer
+            if (lane == 0) {
+                const uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
+                TileCursor cur;
+                cur.seek(p, sh, t_begin);
+                uint32_t tile_no = 0;      // tiles of this block so far (ring position)
+                uint32_t ug = 0;           // global unit counter: unit = (tile, row group)
+                uint32_t seg_no = 0;
+                bool ok = true;
+                for (long long tg = t_begin; tg < t_end && ok;) {
+                    const int seg_tiles = (int)min((long long)(cur.n_tiles - cur.t), t_end - tg);
+                    const int n_units = seg_tiles * NQ;
+                    ok = bounded_wait(smem_u32(&sh->q_full), seg_no & 1, sh, p.device_status);
+                    tc_fence_after();
+                    auto issue_qk = [&](int u) {       // unit u of this segment
+                        const int q = u % NQ, ti = u / NQ;
+                        const uint32_t item = 2 * (tile_no + ti);
+                        const uint32_t slot = item % (uint32_t)n_slots;
+                        if (q == 0) {
+                            ok = ok && bounded_wait(smem_u32(&sh->full[slot]), (item / n_slots) & 1, sh,
+                                                    p.device_status);
+                            tc_fence_after();
+                        }
+                        if (!ok) return;
+                        const uint32_t ka = smem_u32(ring + slot * SLOT_BYTES);
+                        const uint32_t qa = smem_u32(q_smem + q * QGROUP_BYTES);
+                        const uint32_t d = tmem + ((ug + u) & 1) * 128;
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            const uint32_t off = (ks >> 2) * (SLOT_BYTES / 2) + (ks & 3) * 32;
+                            tc_mma_ss(d, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024),
+                                      idesc_qk, ks > 0);
+                        }
+                        tc_commit(smem_u32(&sh->s_full[(ug + u) & 1]));
+                        if (q == NQ - 1) tc_commit(smem_u32(&sh->empty[slot]));   // K tile consumed
+                    };
+                    issue_qk(0);
+                    if (n_units > 1) issue_qk(1);
+                    for (int u = 0; u < n_units && ok; ++u) {
+                        const int q = u % NQ, ti = u / NQ;
+                        const uint32_t gu = ug + u;
+                        ok = bounded_wait(smem_u32(&sh->p_full[gu & 1]), (gu >> 1) & 1, sh, p.device_status);
+                        const uint32_t item = 2 * (tile_no + ti) + 1;
+                        const uint32_t slot = item % (uint32_t)n_slots;
+                        if (ok && q == 0)
+                            ok = bounded_wait(smem_u32(&sh->full[slot]), (item / n_slots) & 1, sh,
+                                              p.device_status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t va = smem_u32(ring + slot * SLOT_BYTES);
+                        const uint32_t pa = tmem + (gu & 1) * 128;       // P overlays S, 64 columns
+                        const uint32_t d = tmem + 256 + q * 128;
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks)
+                            tc_mma_ts(d, pa + ks * 8, smem_desc(va + ks * 2048, SLOT_BYTES / 2, 1024),
+                                      idesc_pv, (ti > 0 || ks > 0) ? 1u : 0u);
+                        tc_commit(smem_u32(&sh->o_done[q]));
+                        if (q == NQ - 1) tc_commit(smem_u32(&sh->empty[slot]));   // V tile consumed
+                        if (u + 2 < n_units) issue_qk(u + 2);
+                    }
+                    ug += n_units;
+                    tile_no += seg_tiles;
+                    ++seg_no;
+                    tg += seg_tiles;
+                    cur.t += seg_tiles;
+                    if (cur.t == cur.n_tiles) cur.next_pair(p);
+                }
+            }
+        } else if (warp >= 4 && warp < 4 + 4 * NQ) {
+            // ================================================================ softmax / epilogue
+            const int q = (warp - 4) >> 2;                     // row group of this warp
+            const int quarter = warp & 3;
+            const int r_in = quarter * 32 + lane;              // TMEM lane = row inside the group
+            const int r = q * 128 + r_in;                      // row of the (b, g) pair
+            const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+            TileCursor cur;
+            cur.seek(p, sh, t_begin);
+            uint32_t ug = 0, kq = 0;       // global unit counter, units of this group so far
+            uint32_t seg_no = 0;
+            bool ok = true;
+            for (long long tg = t_begin; tg < t_end && ok; ++seg_no) {
+                const int b = cur.b, g = cur.g;
+                const int seg_tiles = (int)min((long long)(cur.n_tiles - cur.t), t_end - tg);
+                const int gam = cur.gam;
+                const int R = gam + 1, L = p.seq_len[b];
+                const int n_rows = G * R;
+                const bool row_ok = r < n_rows;
+                const int i = r / G, hh = r - i * G;
+                const int pos = L - R + i;                     // last visible key of this row
+                const long long q_row = ((long long)p.cu_q[b] + i) * p.hq + (long long)g * G + hh;
+                // ---- this thread's query row -> shared memory (K-major, 128-byte swizzle)
+                {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(
+                        static_cast<const __nv_bfloat16 *>(p.q) + q_row * HD);
+                    uint8_t *dst = q_smem + q * QGROUP_BYTES + r_in * 128;
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const uint4 v = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+                        const int half = c >> 3, chunk = (c & 7) ^ (r_in & 7);
+                        *reinterpret_cast<uint4 *>(dst + half * (QGROUP_BYTES / 2) + chunk * 16) = v;
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    mbar_arrive(smem_u32(&sh->q_full));
+                }
+                float m_ref = -CUDART_INF_F, l_sum = 0.f;
+                const uint32_t o_addr = tmem + lane_addr + 256 + q * 128;
+                for (int ti = 0; ti < seg_tiles && ok; ++ti) {
+                    const uint32_t gu = ug + ti * NQ + q;
+                    const uint32_t s_addr = tmem + lane_addr + (gu & 1) * 128;
+                    ok = bounded_wait(smem_u32(&sh->s_full[gu & 1]), (gu >> 1) & 1, sh, p.device_status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const int tok0 = (cur.t + ti) * TILE;
+                    const bool need_mask = tok0 + TILE - 1 > L - R;    // some row cannot see the whole tile
+                    // pass 1: row maximum (log2 units)
+                    float m_tile = -CUDART_INF_F;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t s[32];
+                        tc_ld32(s_addr + ch * 32, s);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            float v = __uint_as_float(s[c]);
+                            if (need_mask && tok0 + ch * 32 + c > pos) v = -CUDART_INF_F;
+                            m_tile = fmaxf(m_tile, v);
+                        }
+                    }
+                    m_tile *= c_scale;
+                    float factor = 1.f;
+                    bool rescale = false;
+                    if (m_tile > m_ref + RESCALE_THRESHOLD || m_ref == -CUDART_INF_F) {
+                        if (m_tile > -CUDART_INF_F) {
+                            rescale = (m_ref > -CUDART_INF_F);
+                            factor = rescale ? ex2_approx(m_ref - m_tile) : 1.f;
+                            m_ref = m_tile;
+                        }
+                    }
+                    const float m_use = (m_ref == -CUDART_INF_F) ? 0.f : m_ref;
+                    // previous PV of this row group must be complete before O may be touched;
+                    // waiting every time keeps the barrier's phase in step with kq
+                    if (kq > 0) ok = bounded_wait(smem_u32(&sh->o_done[q]), (kq - 1) & 1, sh, p.device_status);
+                    if (!ok) break;
+                    if (rescale) l_sum *= factor;
+                    // tensor-memory accesses are warp-wide: if any row of the warp has to rescale
+                    // its accumulator, the whole warp goes through (factor 1 elsewhere)
+                    if (__any_sync(0xffffffffu, rescale && ti > 0)) {
+                        tc_fence_after();
+                        const float f = (rescale && ti > 0) ? factor : 1.f;
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            uint32_t o[32];
+                            tc_ld32(o_addr + ch * 32, o);
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
+                            tc_st32(o_addr + ch * 32, o);
+                        }
+                    }
+                    // pass 2: P = 2^(s*c - m_ref) as bf16 pairs, written over S
+                    float tile_sum = 0.f;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        float chunk_sum = 0.f;
+                        uint32_t s[32];
+                        tc_ld32(s_addr + ch * 32, s);
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int c = 0; c < 32; c += 2) {
+                            float e0 = ex2_approx(fmaf(__uint_as_float(s[c]), c_scale, -m_use));
+                            float e1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), c_scale, -m_use));
+                            if (need_mask) {
+                                if (tok0 + ch * 32 + c > pos) e0 = 0.f;
+                                if (tok0 + ch * 32 + c + 1 > pos) e1 = 0.f;
+                            }
+                            chunk_sum += e0 + e1;
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(e0, e1);
+                            pk[c >> 1] = *reinterpret_cast<const uint32_t *>(&h);
+                        }
+                        tile_sum += chunk_sum;
+                        // 16 packed columns: chunk ch of P goes to columns [16 ch, 16 ch + 16) of the
+                        // S buffer, which lie inside S chunks that have already been read.
+                        asm volatile(
+                            "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+                            "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(
+                                s_addr + ch * 16),
+                            "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]),
+                            "r"(pk[7]), "r"(pk[8]), "r"(pk[9]), "r"(pk[10]), "r"(pk[11]), "r"(pk[12]),
+                            "r"(pk[13]), "r"(pk[14]), "r"(pk[15])
+                            : "memory");
+                    }
+                    l_sum += tile_sum;
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&sh->p_full[gu & 1]));
+                    ++kq;
+                }
+                if (!ok) break;
+                // ---- epilogue of the segment: wait for the last PV, then read O
+                ok = bounded_wait(smem_u32(&sh->o_done[q]), (kq - 1) & 1, sh, p.device_status);
+                if (!ok) break;
+                tc_fence_after();
+                const bool whole = (cur.t == 0 && seg_tiles == cur.n_tiles);
+                if (whole) {
+                    const float inv = 1.f / l_sum;
+                    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.o) + q_row * HD;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t o[32];
+                        tc_ld32(o_addr + ch * 32, o);
+                        if (row_ok) {
+#pragma unroll
+                            for (int c = 0; c < 32; c += 8) {
+                                uint4 w;
+                                uint32_t *wp = reinterpret_cast<uint32_t *>(&w);
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const __nv_bfloat162 h = __floats2bfloat162_rn(
+                                        __uint_as_float(o[c + 2 * e]) * inv, __uint_as_float(o[c + 2 * e + 1]) * inv);
+                                    wp[e] = *reinterpret_cast<const uint32_t *>(&h);
+                                }
+                                *reinterpret_cast<uint4 *>(dst + ch * 32 + c) = w;
+                            }
+                        }
+                    }
+                    if (row_ok && p.lse != nullptr)
+                        p.lse[q_row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+                } else {
+                    // partial: fp32 O row, then max and sum; slot 0 = the block's first segment
+                    float *slot = a.ws_part + ((size_t)blockIdx.x * 2 + (seg_no == 0 ? 0 : 1)) * part_slot_floats(NQ);
+                    float *orow = slot + (size_t)r * HD;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t o[32];
+                        tc_ld32(o_addr + ch * 32, o);
+                        if (row_ok) {
+#pragma unroll
+                            for (int c = 0; c < 32; c += 4)
+                                *reinterpret_cast<uint4 *>(orow + ch * 32 + c) = make_uint4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+                        }
+                    }
+                    if (row_ok) {
+                        slot[(size_t)NQ * 128 * HD + r] = m_ref;
+                        slot[(size_t)NQ * 128 * HD + NQ * 128 + r] = l_sum;
+                    }
+                }
+                tc_fence_before();
+                ug += seg_tiles * NQ;
+                tg += seg_tiles;
+                cur.t += seg_tiles;
+                if (cur.t == cur.n_tiles) cur.next_pair(p);
+            }
+        }
+    }
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------- combine kernel
+// One block per (sequence, kv head); merges the partials of pairs whose tiles were shared
+// by several blocks of the main kernel.  Thread = query row.
+__global__ void __launch_bounds__(256)
+attn_combine_kernel(const AttnTcLaunch a)
+{
+    const sv_attn_params &p = a.p;
+    const int b = blockIdx.x / p.hkv, g = blockIdx.x % p.hkv;
+    const int NQ = a.nq;
+    const long long grid = a.ws_prefix[p.batch + 1];
+    const long long total = (long long)a.ws_prefix[p.batch] * p.hkv;
+    const int n_tiles = a.ws_prefix[b + 1] - a.ws_prefix[b];
+    if (n_tiles == 0 || total == 0) return;
+    const long long T0 = (long long)a.ws_prefix[b] * p.hkv + (long long)g * n_tiles, T1 = T0 + n_tiles;
+    // blocks whose share contains tile T0 and tile T1-1
+    const long long c_first = ((T0 + 1) * grid + total - 1) / total - 1;
+    const long long c_last = (T1 * grid + total - 1) / total - 1;
+    if (c_first == c_last && share_begin(c_first, total, grid) <= T0 &&
+        share_begin(c_first + 1, total, grid) >= T1)
+        return;                                          // one block saw the whole pair: already final
+    int gam = p.gamma[b];
+    gam = min(max(gam, 0), p.gamma_max);
+    const int G = a.group, n_rows = G * (gam + 1);
+    for (int r = threadIdx.x; r < n_rows; r += blockDim.x) {
+        float m = -CUDART_INF_F;
+        for (long long c = c_first; c <= c_last; ++c) {
+            if (share_begin(c + 1, total, grid) == share_begin(c, total, grid)) continue;   // empty share
+            const int which = (share_begin(c, total, grid) >= T0) ? 0 : 1;
+            const float *slot = a.ws_part + ((size_t)c * 2 + which) * part_slot_floats(NQ);
+            m = fmaxf(m, slot[(size_t)NQ * 128 * HD + r]);
+        }
+        float acc[HD];
+#pragma unroll
+        for (int d = 0; d < HD; ++d) acc[d] = 0.f;
+        float l = 0.f;
+        for (long long c = c_first; c <= c_last; ++c) {
+            if (share_begin(c + 1, total, grid) == share_begin(c, total, grid)) continue;
+            const int which = (share_begin(c, total, grid) >= T0) ? 0 : 1;
+            const float *slot = a.ws_part + ((size_t)c * 2 + which) * part_slot_floats(NQ);
+            const float mc = slot[(size_t)NQ * 128 * HD + r];
+            if (mc == -CUDART_INF_F) continue;
+            const float w = exp2f(mc - m);
+            l += w * slot[(size_t)NQ * 128 * HD + NQ * 128 + r];
+            const float4 *orow = reinterpret_cast<const float4 *>(slot + (size_t)r * HD);
+#pragma unroll
+            for (int d = 0; d < HD / 4; ++d) {
+                const float4 v = orow[d];
+                acc[4 * d] += w * v.x; acc[4 * d + 1] += w * v.y;
+                acc[4 * d + 2] += w * v.z; acc[4 * d + 3] += w * v.w;
+            }
+        }
+        const int i = r / G, hh = r - i * G;
+        const long long q_row = ((long long)p.cu_q[b] + i) * p.hq + (long long)g * G + hh;
+        const float inv = 1.f / l;
+        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.o) + q_row * HD;
+#pragma unroll
+        for (int d = 0; d < HD; d += 2)
+            *reinterpret_cast<__nv_bfloat162 *>(dst + d) = __floats2bfloat162_rn(acc[d] * inv, acc[d + 1] * inv);
+        if (p.lse != nullptr) p.lse[q_row] = (m + log2f(l)) * 0.6931471805599453f;
+    }
+}
+
+// ---------------------------------------------------------------------------- host side
+static int rows_groups(const sv_attn_params &p)
+{
+    const int rows = (p.hq / p.hkv) * (p.gamma_max + 1);
+    return (rows + 127) / 128;
+}
+
+bool attn_tc_supported(const sv_attn_params &p)
+{
+    if (p.head_dim != HD || p.pool == nullptr || !p.pool->has_maps) return false;
+    if (p.batch > MAX_BATCH_TC) return false;
+    const int nq = rows_groups(p);
+    return nq >= 1 && nq <= 2;
+}
+
+static size_t prefix_bytes(int batch) { return (((size_t)batch + 2) * sizeof(int32_t) + 255) & ~(size_t)255; }
+
+size_t attn_tc_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t hq, int32_t hkv,
+                               int32_t head_dim, int32_t max_seq_len)
+{
+    (void)max_seq_len;
+    if (head_dim != HD || hkv <= 0 || hq % hkv != 0) return 0;
+    const int rows = (hq / hkv) * (gamma_max + 1);
+    const int nq = (rows + 127) / 128;
+    if (nq < 1 || nq > 2 || batch > MAX_BATCH_TC) return 0;
+    return prefix_bytes(batch) + (size_t)sm_count() * 2 * part_slot_floats(nq) * sizeof(float);
+}
+
+sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t workspace_bytes,
+                         cudaStream_t stream)
+{
+    AttnTcLaunch a;
+    a.p = p;
+    a.n_pool_pages = p.pool->n_pages;
+    a.group = p.hq / p.hkv;
+    a.nq = rows_groups(p);
+    const int grid = sm_count();
+    if (workspace_bytes < prefix_bytes(p.batch) + (size_t)grid * 2 * part_slot_floats(a.nq) * sizeof(float))
+        return SV_EWORKSPACE;
+    a.ws_prefix = static_cast<int32_t *>(workspace);
+    a.ws_part = reinterpret_cast<float *>(static_cast<uint8_t *>(workspace) + prefix_bytes(p.batch));
+    const size_t fixed = (size_t)a.nq * QGROUP_BYTES + sizeof(Shared) + 1024;
+    const size_t budget = 227 * 1024;
+    a.n_slots = (int)((budget - fixed) / SLOT_BYTES);
+    if (a.n_slots > 8) a.n_slots = 8;
+    if (a.n_slots < 4) return SV_EUNSUPPORTED;
+    const size_t smem = fixed + (size_t)a.n_slots * SLOT_BYTES;
+    cudaError_t e;
+    if (a.nq == 1) {
+        e = cudaFuncSetAttribute(attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return SV_ECUDA;
+        attn_tc_kernel<1><<<grid, 256, smem, stream>>>(a, p.pool->k_map, p.pool->v_map);
+    } else {
+        e = cudaFuncSetAttribute(attn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return SV_ECUDA;
+        attn_tc_kernel<2><<<grid, 384, smem, stream>>>(a, p.pool->k_map, p.pool->v_map);
+    }
+    sv_status st = launch_check();
+    if (st != SV_OK) return st;
+    attn_combine_kernel<<<p.batch * p.hkv, 256, 0, stream>>>(a);
+    return launch_check();
+}
+
+}  // namespace sv

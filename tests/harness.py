@@ -88,6 +88,16 @@ def used_rows(gamma, cu_q):
 
 
 ATTN_ATOL = 2e-2        # bf16 attention outputs, absolute
+
+
+def attn_allowed(o_ref):
+    """2e-2 absolute.  A bf16 value of magnitude >= 4 is a multiple of 2^-5, so its correctly
+    rounded result can already sit 0.0156 from the exact one; for those elements (reached only
+    by the peaky stress cases) half a bf16 ulp of the reference is added to the bound."""
+    a = np.abs(o_ref)
+    return ATTN_ATOL + np.where(a >= 4.0, a * 2.0 ** -8, 0.0)
+
+
 SUM_RTOL = 1e-5         # fp32 softmax sums, relative
 
 
@@ -96,8 +106,11 @@ def check_attn(case: AttnCase):
     o_ref, lse_ref = run_attn_oracle(case)
     rows = used_rows(case.gamma, case.cu_q)
     assert status == 0, f"device status {status}"
-    err = np.abs(o_gpu[rows] - o_ref[rows]).max()
-    assert err <= ATTN_ATOL, f"attention output error {err}"
+    diff = np.abs(o_gpu[rows] - o_ref[rows])
+    err = diff.max()
+    w = np.unravel_index(np.argmax(diff - attn_allowed(o_ref[rows])), diff.shape)
+    assert (diff <= attn_allowed(o_ref[rows])).all(), \
+        f"attention output error {diff[w]} at used-row {w}: gpu {o_gpu[rows][w]} vs oracle {o_ref[rows][w]}"
     # softmax sums: exp(lse) relative error
     rel = np.abs(np.expm1(lse_gpu[rows] - lse_ref[rows])).max()
     assert rel <= SUM_RTOL, f"softmax sum relative error {rel}"
