@@ -118,6 +118,22 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
         : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// same without the wait: several loads can be in flight, then one tc_wait_ld()
+__device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t *r)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+          "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+          "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+          "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32])
 {
     asm volatile(
@@ -346,8 +362,11 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
     const uint32_t tmem = sh->tmem_base;
     const float c_scale = p.sm_scale * 1.4426950408889634f;   // scores in log2 units
 
-    if (t_end > t_begin) {
-        if (warp == 0) {
+    // With two row groups there are 384 threads and 168 registers each; the producer / MMA
+    // warpgroup hands part of its share to the softmax warpgroups (128*80 + 256*208 <= 384*168).
+    if (warp < 4) {
+        if (NQ == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+        if (t_end > t_begin && warp == 0) {
             // ================================================================ TMA producer
             TileCursor cur;
             cur.seek(p, sh, t_begin);
@@ -387,7 +406,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 if (!ok) break;
                 if (++cur.t == cur.n_tiles) cur.next_pair(p);
             }
-        } else if (warp == 1) {
+        } else if (t_end > t_begin && warp == 1) {
             // ================================================================ MMA issuer
             if (lane == 0) {
                 const uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
@@ -399,11 +418,13 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 bool ok = true;
                 for (long long tg = t_begin; tg < t_end && ok;) {
                     const int seg_tiles = (int)min((long long)(cur.n_tiles - cur.t), t_end - tg);
-                    const int n_units = seg_tiles * NQ;
+                    // row groups this pair really has (a second group only if it has > 128 rows)
+                    const int nq_seg = (NQ == 2 && G * (cur.gam + 1) > 128) ? 2 : 1;
+                    const int n_units = seg_tiles * nq_seg;
                     ok = bounded_wait(smem_u32(&sh->q_full), seg_no & 1, sh, p.device_status);
                     tc_fence_after();
                     auto issue_qk = [&](int u) {       // unit u of this segment
-                        const int q = u % NQ, ti = u / NQ;
+                        const int q = u % nq_seg, ti = u / nq_seg;
                         const uint32_t item = 2 * (tile_no + ti);
                         const uint32_t slot = item % (uint32_t)n_slots;
                         if (q == 0) {
@@ -422,12 +443,12 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                                       idesc_qk, ks > 0);
                         }
                         tc_commit(smem_u32(&sh->s_full[(ug + u) & 1]));
-                        if (q == NQ - 1) tc_commit(smem_u32(&sh->empty[slot]));   // K tile consumed
+                        if (q == nq_seg - 1) tc_commit(smem_u32(&sh->empty[slot]));   // K tile consumed
                     };
                     issue_qk(0);
                     if (n_units > 1) issue_qk(1);
                     for (int u = 0; u < n_units && ok; ++u) {
-                        const int q = u % NQ, ti = u / NQ;
+                        const int q = u % nq_seg, ti = u / nq_seg;
                         const uint32_t gu = ug + u;
                         ok = bounded_wait(smem_u32(&sh->p_full[gu & 1]), (gu >> 1) & 1, sh, p.device_status);
                         const uint32_t item = 2 * (tile_no + ti) + 1;
@@ -445,7 +466,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                             tc_mma_ts(d, pa + ks * 8, smem_desc(va + ks * 2048, SLOT_BYTES / 2, 1024),
                                       idesc_pv, (ti > 0 || ks > 0) ? 1u : 0u);
                         tc_commit(smem_u32(&sh->o_done[q]));
-                        if (q == NQ - 1) tc_commit(smem_u32(&sh->empty[slot]));   // V tile consumed
+                        if (q == nq_seg - 1) tc_commit(smem_u32(&sh->empty[slot]));   // V tile consumed
                         if (u + 2 < n_units) issue_qk(u + 2);
                     }
                     ug += n_units;
@@ -456,7 +477,10 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     if (cur.t == cur.n_tiles) cur.next_pair(p);
                 }
             }
-        } else if (warp >= 4 && warp < 4 + 4 * NQ) {
+        }
+    } else {
+        if (NQ == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+        if (t_end > t_begin) {
             // ================================================================ softmax / epilogue
             const int q = (warp - 4) >> 2;                     // row group of this warp
             const int quarter = warp & 3;
@@ -474,12 +498,15 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 const int gam = cur.gam;
                 const int R = gam + 1, L = p.seq_len[b];
                 const int n_rows = G * R;
+                const int nq_seg = (NQ == 2 && n_rows > 128) ? 2 : 1;
+                const bool grp_active = q < nq_seg;                       // this row group exists for the pair
+                const bool warp_active = grp_active && (q * 128 + quarter * 32 < n_rows);
                 const bool row_ok = r < n_rows;
                 const int i = r / G, hh = r - i * G;
                 const int pos = L - R + i;                     // last visible key of this row
                 const long long q_row = ((long long)p.cu_q[b] + i) * p.hq + (long long)g * G + hh;
                 // ---- this thread's query row -> shared memory (K-major, 128-byte swizzle)
-                {
+                if (grp_active) {
                     const uint4 *src = reinterpret_cast<const uint4 *>(
                         static_cast<const __nv_bfloat16 *>(p.q) + q_row * HD);
                     uint8_t *dst = q_smem + q * QGROUP_BYTES + r_in * 128;
@@ -490,32 +517,49 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                         *reinterpret_cast<uint4 *>(dst + half * (QGROUP_BYTES / 2) + chunk * 16) = v;
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    mbar_arrive(smem_u32(&sh->q_full));
+                }
+                mbar_arrive(smem_u32(&sh->q_full));
+                if (!grp_active) {                              // nothing to do for this pair
+                    ug += seg_tiles * nq_seg;
+                    tg += seg_tiles;
+                    cur.t += seg_tiles;
+                    if (cur.t == cur.n_tiles) cur.next_pair(p);
+                    continue;
                 }
                 float m_ref = -CUDART_INF_F, l_sum = 0.f;
                 const uint32_t o_addr = tmem + lane_addr + 256 + q * 128;
                 for (int ti = 0; ti < seg_tiles && ok; ++ti) {
-                    const uint32_t gu = ug + ti * NQ + q;
+                    const uint32_t gu = ug + ti * nq_seg + q;
                     const uint32_t s_addr = tmem + lane_addr + (gu & 1) * 128;
                     ok = bounded_wait(smem_u32(&sh->s_full[gu & 1]), (gu >> 1) & 1, sh, p.device_status);
                     if (!ok) break;
+                    if (!warp_active) {                         // all 32 rows are padding
+                        mbar_arrive(smem_u32(&sh->p_full[gu & 1]));
+                        ++kq;
+                        continue;
+                    }
                     tc_fence_after();
                     const int tok0 = (cur.t + ti) * TILE;
                     const bool need_mask = tok0 + TILE - 1 > L - R;    // some row cannot see the whole tile
-                    // pass 1: row maximum (log2 units)
-                    float m_tile = -CUDART_INF_F;
+                    // the row's 128 scores: four loads in flight, one wait
+                    uint32_t s[128];
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        uint32_t s[32];
-                        tc_ld32(s_addr + ch * 32, s);
+                    for (int ch = 0; ch < 4; ++ch) tc_ld32_nowait(s_addr + ch * 32, s + ch * 32);
+                    tc_wait_ld();
+                    if (need_mask) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            float v = __uint_as_float(s[c]);
-                            if (need_mask && tok0 + ch * 32 + c > pos) v = -CUDART_INF_F;
-                            m_tile = fmaxf(m_tile, v);
-                        }
+                        for (int c = 0; c < 128; ++c)
+                            if (tok0 + c > pos) s[c] = 0xff800000u;     // -inf
                     }
-                    m_tile *= c_scale;
+                    float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
+#pragma unroll
+                    for (int c = 0; c < 128; c += 4) {
+                        m0 = fmaxf(m0, __uint_as_float(s[c]));
+                        m1 = fmaxf(m1, __uint_as_float(s[c + 1]));
+                        m2 = fmaxf(m2, __uint_as_float(s[c + 2]));
+                        m3 = fmaxf(m3, __uint_as_float(s[c + 3]));
+                    }
+                    const float m_tile = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * c_scale;
                     float factor = 1.f;
                     bool rescale = false;
                     if (m_tile > m_ref + RESCALE_THRESHOLD || m_ref == -CUDART_INF_F) {
@@ -545,29 +589,23 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                             tc_st32(o_addr + ch * 32, o);
                         }
                     }
-                    // pass 2: P = 2^(s*c - m_ref) as bf16 pairs, written over S
+                    // P = 2^(s*c - m_ref) as bf16 pairs, written over S (masked scores are -inf -> 0)
                     float tile_sum = 0.f;
 #pragma unroll
                     for (int ch = 0; ch < 4; ++ch) {
-                        float chunk_sum = 0.f;
-                        uint32_t s[32];
-                        tc_ld32(s_addr + ch * 32, s);
+                        float sum0 = 0.f, sum1 = 0.f;
                         uint32_t pk[16];
 #pragma unroll
                         for (int c = 0; c < 32; c += 2) {
-                            float e0 = ex2_approx(fmaf(__uint_as_float(s[c]), c_scale, -m_use));
-                            float e1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), c_scale, -m_use));
-                            if (need_mask) {
-                                if (tok0 + ch * 32 + c > pos) e0 = 0.f;
-                                if (tok0 + ch * 32 + c + 1 > pos) e1 = 0.f;
-                            }
-                            chunk_sum += e0 + e1;
+                            const float e0 = ex2_approx(fmaf(__uint_as_float(s[ch * 32 + c]), c_scale, -m_use));
+                            const float e1 = ex2_approx(fmaf(__uint_as_float(s[ch * 32 + c + 1]), c_scale, -m_use));
+                            sum0 += e0;
+                            sum1 += e1;
                             const __nv_bfloat162 h = __floats2bfloat162_rn(e0, e1);
                             pk[c >> 1] = *reinterpret_cast<const uint32_t *>(&h);
                         }
-                        tile_sum += chunk_sum;
-                        // 16 packed columns: chunk ch of P goes to columns [16 ch, 16 ch + 16) of the
-                        // S buffer, which lie inside S chunks that have already been read.
+                        tile_sum += sum0 + sum1;
+                        // chunk ch of P: 16 packed columns at [16 ch, 16 ch + 16) of the S buffer
                         asm volatile(
                             "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
                             "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(
@@ -589,7 +627,9 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 if (!ok) break;
                 tc_fence_after();
                 const bool whole = (cur.t == 0 && seg_tiles == cur.n_tiles);
-                if (whole) {
+                if (!warp_active) {
+                    // padding rows: nothing to write
+                } else if (whole) {
                     const float inv = 1.f / l_sum;
                     __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.o) + q_row * HD;
 #pragma unroll
@@ -633,7 +673,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     }
                 }
                 tc_fence_before();
-                ug += seg_tiles * NQ;
+                ug += seg_tiles * nq_seg;
                 tg += seg_tiles;
                 cur.t += seg_tiles;
                 if (cur.t == cur.n_tiles) cur.next_pair(p);
