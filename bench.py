@@ -45,8 +45,10 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
 
 
-def workload_inputs(cfg, rank, batch=None):
+def workload_inputs(cfg, rank, batch=None, gamma=None):
     cfg = synth.scaled(cfg, seed=cfg.seed + 1000 * rank)
+    if gamma is not None:
+        cfg = synth.scaled(cfg, gamma_lo=gamma, gamma_hi=gamma)
     if batch:
         cfg = synth.scaled(cfg, batch=batch)
     seq_len, gamma = synth.draw_lengths(cfg)
@@ -89,7 +91,7 @@ def run_reference(args):
         return
     import oracle
     oracle.build()
-    cfg, seq_len, gamma, cu_q, cu_d = workload_inputs(synth.CONFIGS[args.workload], 0, args.batch)
+    cfg, seq_len, gamma, cu_q, cu_d = workload_inputs(synth.CONFIGS[args.workload], 0, args.batch, args.gamma)
     n_seq = min(args.oracle_seqs or 4, cfg.batch)
     sub, kv, q, li = sample_inputs(cfg, seq_len, gamma, cu_q, cu_d, n_seq)
     times, toks = [], 0
@@ -187,7 +189,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(DEV))
 
     base_cfg = synth.CONFIGS[args.workload]
-    cfg, seq_len, gamma, cu_q, cu_d = workload_inputs(base_cfg, rank, args.batch)
+    cfg, seq_len, gamma, cu_q, cu_d = workload_inputs(base_cfg, rank, args.batch, args.gamma)
     B, gmax = cfg.batch, cfg.gamma_max
     n_q, n_d = int(cu_q[-1]), int(cu_d[-1])
     kv = synth.make_kv(cfg, seq_len, reserve_tokens=2 * (gmax + 1))
@@ -384,6 +386,8 @@ def main():
                     help="sequences in the oracle's bounded sample (default 16 for cpu_baseline, 4 per step for --impl reference)")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--gamma", type=int, default=None,
+                    help="draft length of every sequence (default: the workload's own range)")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the workload's batch (smaller cases for profiler captures)")
     args = ap.parse_args()

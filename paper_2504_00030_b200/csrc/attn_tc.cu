@@ -520,6 +520,14 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 }
                 mbar_arrive(smem_u32(&sh->q_full));
                 if (!grp_active) {                              // nothing to do for this pair
+                    // Stay in step with the barriers this group will use again later: a parity
+                    // wait is only meaningful for a waiter that is at most one phase ahead, so the
+                    // idle group follows every phase of q_full and of both s_full barriers.
+                    ok = bounded_wait(smem_u32(&sh->q_full), seg_no & 1, sh, p.device_status);
+                    for (int ti = 0; ti < seg_tiles && ok; ++ti) {
+                        const uint32_t gu = ug + ti;            // nq_seg == 1 here
+                        ok = bounded_wait(smem_u32(&sh->s_full[gu & 1]), (gu >> 1) & 1, sh, p.device_status);
+                    }
                     ug += seg_tiles * nq_seg;
                     tg += seg_tiles;
                     cur.t += seg_tiles;

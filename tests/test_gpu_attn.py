@@ -55,6 +55,16 @@ def test_ragged_gqa_many_sequences():
     check_attn(make_attn_case(cfg))
 
 
+def test_mixed_row_counts_around_128():
+    # 8 query heads per kv head, gamma from 0 to 16: pairs with 8 .. 136 rows in one launch,
+    # so pairs that need the second row group alternate with pairs that do not
+    cfg = synth.VerifyConfig("mixed", 20, 16, 2, 128, 100, 100, 1800, 0, 16, 16, 1.0, 1.0, q_scale=3.0,
+                             seed=50)
+    gamma = np.array([16, 15, 16, 0, 7, 16, 16, 14, 15, 16, 1, 16, 15, 15, 16, 3, 16, 16, 15, 2], np.int32)
+    check_attn(make_attn_case(cfg, gamma=gamma))
+    check_attn(make_attn_case(cfg, gamma=np.full(20, 15, np.int32)))
+
+
 def test_long_context_single_sequence():
     cfg = synth.VerifyConfig("long", 1, 8, 1, 128, 100, 16384, 16384, 16, 16, 16, 1.0, 1.0, q_scale=6.0,
                              seed=44)
