@@ -181,12 +181,14 @@ sv_status spec_accept_sample(const sv_accept_params *p, void *workspace_device,
  * differs: they go to an array of SV_ACCEPT_STATIC_SCRATCH_BYTES bytes that is
  * built into the library (each GPU that loads the library carries it until the
  * process ends).
- *   - Limit: batch * (2*gamma_max + 1) * slices * 32 bytes must not exceed
- *     SV_ACCEPT_STATIC_SCRATCH_BYTES, where slices = ceil(vocab / slice) and the
- *     library picks slice between 2048 and 16384 elements (larger when there are
- *     many rows).  The largest configuration of the tests (batch 128, gamma_max
- *     16, vocab 128256) needs about 1.1 MB.  A larger problem is refused with
- *     SV_EWORKSPACE before anything is launched; use spec_accept_sample then.
+ *   - Limit: the intermediate results -- 32 bytes per (row, slice of the
+ *     vocabulary) with batch * (2*gamma_max + 1) rows and slices of 2048 to 16384
+ *     elements (the library picks larger slices when there are many rows), plus
+ *     24 bytes per 128 vocabulary entries per sequence for the sampling pass --
+ *     must fit in SV_ACCEPT_STATIC_SCRATCH_BYTES.  The largest configuration of
+ *     the tests (batch 128, gamma_max 16, vocab 128256) needs about 4.2 MB.  A
+ *     larger problem is refused with SV_EWORKSPACE before anything is launched;
+ *     use spec_accept_sample then.
  *   - The first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress) with that device current; make that first call
  *     outside any stream capture.  No call allocates or frees memory.
@@ -197,7 +199,7 @@ sv_status spec_accept_sample(const sv_accept_params *p, void *workspace_device,
  *     array and give wrong results; keep such calls on one stream or order them
  *     with events.
  */
-#define SV_ACCEPT_STATIC_SCRATCH_BYTES (4u << 20)
+#define SV_ACCEPT_STATIC_SCRATCH_BYTES (8u << 20)
 sv_status spec_accept_sample_static(const sv_accept_params *p, void *stream);
 
 /* ---------------------------------------------------------------- GammaTune */

@@ -290,7 +290,7 @@ def spec_accept_sample(target_logits, draft_logits, draft_tokens, u_accept, u_sa
                                      _stream(stream)))
 
 
-SV_ACCEPT_STATIC_SCRATCH_BYTES = 4 << 20
+SV_ACCEPT_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 def spec_accept_sample_static(target_logits, draft_logits, draft_tokens, u_accept, u_sample, temperature,

@@ -1,33 +1,35 @@
 // Fused speculative-sampling acceptance over the vocabulary (paper Section 3).
 //
-// Two kernels per step:
+// Four kernels per step, all on the caller's stream:
 //
-//  1. accept_rowstats_kernel -- the streaming pass.  Every target and draft
-//     logit is read exactly once with 128-bit loads; for each (row, slice of the
-//     vocabulary) one thread block produces the single-pass online softmax
-//     statistics (a power-of-two reference exponent and the sum of
-//     2^(x*log2e/T - ref)) or, for greedy sequences, the (max, lowest index).
-//     Exponentials are float32 (ex2.approx); sums are carried in float64 and
-//     every rescale is by an exact power of two, so the only error in a row's
-//     partition function is the per-element float32 rounding.
-//
-//  2. accept_finish_kernel -- one thread block per sequence: merges the slice
-//     statistics into ln Z per row, evaluates ratio_i = min(1, p_i[x_i]/q_i[x_i])
-//     and the comparison with u_i in float64, finds the first rejection, and
-//     draws the next token from the residual max(0, p_n - q_n) (or the bonus
-//     row) by inverse CDF.  That last part re-reads only the one or two rows it
-//     samples from and works entirely in float64.
+//  1. accept_rowstats_kernel -- the streaming pass and the only one that touches every
+//     logit.  Each (row, slice of the vocabulary) item is owned by ONE WARP: 128-bit
+//     streaming loads, eight per lane in flight, a single-pass online softmax with a
+//     power-of-two running reference (so every rescale is exact), float32 ex2.approx
+//     exponentials summed four at a time into a float64 accumulator, and a warp-shuffle
+//     reduction at the end.  No block-level synchronisation at all.  Greedy sequences
+//     (T = 0) only track (max, lowest index) of their target rows.
+//  2. accept_decide_kernel -- one block per sequence: merges the slice statistics into
+//     ln Z per row (float64), evaluates ratio_i = min(1, p_i[x_i]/q_i[x_i]) against u_i in
+//     float64 for all positions in parallel, then takes the first rejection.
+//  3. accept_segsum_kernel -- float64 pass over the one or two rows the next token is
+//     drawn from (residual max(0, p_n - q_n) or the bonus row): sums per 128-token
+//     segment, the sign of p_k - q_k decided with the first-pass partition sums.
+//  4. accept_pick_kernel -- one warp per sequence: exact partition sums, inverse CDF over
+//     the segment sums, exact float64 resolution inside the chosen segment.
 #include "common.cuh"
 
 #include <math_constants.h>
 
 namespace sv {
 
-constexpr int RS_THREADS = 256;   // rowstats block
-constexpr int RS_UNROLL = 4;      // float4 loads in flight per thread
-constexpr int FIN_THREADS = 512;  // finish block
+constexpr int RS_THREADS = 256;   // rowstats block (8 independent warps)
+constexpr int RS_UNROLL = 8;      // float4 loads in flight per lane
 constexpr int SEG = 128;          // vocabulary elements per sampling segment (one warp, float4 per lane)
+constexpr int SEG_THREADS = 256;
+constexpr int MAX_SPLITS = 16;    // blocks per sequence in the segment-sum pass
 constexpr int MIN_SLICE = 2048;
+constexpr int MAX_SLICE = 16384;
 constexpr float REF_INIT = -1.0e30f;
 
 struct __align__(16) RowPartial {
@@ -38,12 +40,25 @@ struct __align__(16) RowPartial {
     int32_t pad;
 };
 
+// what the decision kernel leaves for the sampling kernels, one per sequence
+struct __align__(16) SeqRecord {
+    double sum_p_hat, sum_q_hat;  // first-pass sums of the sampled rows (at ref_p / ref_q)
+    float ref_p, ref_q;
+    int32_t n;                    // first rejection (gamma if none)
+    int32_t mode;                 // 0: nothing to sample (greedy or failed), 1: residual, 2: bonus row
+};
+
 struct AcceptLaunch {
     sv_accept_params p;
-    RowPartial *partials;
-    int slice;       // elements per slice (multiple of 1024)
+    RowPartial *partials;   // [batch * (2 gmax + 1) * n_slices]
+    SeqRecord *records;     // [batch]
+    double *seg;            // [batch][3][n_seg]: positive-part sums of a, of b, all of a
+    double *totals;         // [batch][MAX_SPLITS][2]
+    int slice;              // elements per slice (multiple of 1024)
     int n_slices;
-    int vec_ok;      // 128-bit loads legal for every row
+    int n_seg;
+    int splits;
+    int vec_ok;             // 128-bit loads legal for every row
 };
 
 __device__ __forceinline__ float seq_temperature(const sv_accept_params &p, int b)
@@ -61,12 +76,19 @@ __device__ __forceinline__ int seq_gamma(const sv_accept_params &p, int b)
     return g;
 }
 
+// x * 2^k for k <= 0, exact (x >= 0, normal or zero); far below the reference -> 0
+__device__ __forceinline__ double scale_down_pow2(double x, float k)
+{
+    if (!(k > -800.f) || !(x > 0.0)) return (x != x) ? x : 0.0;     // NaN stays NaN
+    if (k == 0.f || x == CUDART_INF) return x;
+    return __hiloint2double(__double2hiint(x) + ((int)k << 20), __double2loint(x));
+}
+
 // (ref, sum) pairs combine by rescaling to the larger reference; the factor is a power of two.
 __device__ __forceinline__ void merge_stats(float &ref, double &sum, float ref2, double sum2)
 {
     const float r = fmaxf(ref, ref2);
-    const float d1 = fmaxf(ref - r, -2000.f), d2 = fmaxf(ref2 - r, -2000.f);
-    sum = scalbn(sum, (int)d1) + scalbn(sum2, (int)d2);
+    sum = scale_down_pow2(sum, ref - r) + scale_down_pow2(sum2, ref2 - r);
     ref = r;
 }
 
@@ -75,8 +97,31 @@ __device__ __forceinline__ void merge_argmax(float &v, int &i, float v2, int i2)
     if (v2 > v || (v2 == v && i2 < i)) { v = v2; i = i2; }
 }
 
+// 2^y in float64 for y <= ~4 (anything below -1000, -inf or NaN gives 0): round to the nearest
+// integer, degree-11 Taylor polynomial of 2^f on [-1/2, 1/2] (error < 1e-14), exponent added
+// by hand.
+__device__ __forceinline__ double exp2_f64(double y)
+{
+    if (!(y > -1000.0)) return 0.0;
+    const double n = rint(y);
+    const double f = y - n;
+    double p = 4.44553827187081e-10;
+    p = fma(p, f, 7.054911620801121e-09);
+    p = fma(p, f, 1.0178086009239696e-07);
+    p = fma(p, f, 1.3215486790144305e-06);
+    p = fma(p, f, 1.5252733804059838e-05);
+    p = fma(p, f, 0.00015403530393381606);
+    p = fma(p, f, 0.0013333558146428441);
+    p = fma(p, f, 0.009618129107628477);
+    p = fma(p, f, 0.055504108664821576);
+    p = fma(p, f, 0.2402265069591007);
+    p = fma(p, f, 0.6931471805599453);
+    p = fma(p, f, 1.0);
+    return __hiloint2double(__double2hiint(p) + ((int)n << 20), __double2loint(p));
+}
+
 // ---------------------------------------------------------------------------------------------
-// Kernel 1: streaming row statistics.
+// Kernel 1: streaming row statistics, one warp per (row, slice).
 // Dense row numbering: sequence b owns rows b*(2*gmax+1) + j; j <= gmax is target row j,
 // j > gmax is draft row j-gmax-1.  Rows a sequence does not have this step are skipped.
 // ---------------------------------------------------------------------------------------------
@@ -86,13 +131,11 @@ accept_rowstats_kernel(AcceptLaunch a)
     const sv_accept_params &p = a.p;
     const int rows_per_seq = 2 * p.gamma_max + 1;
     const long long n_items = (long long)p.batch * rows_per_seq * a.n_slices;
-    __shared__ double s_sum[RS_THREADS / 32];
-    __shared__ float s_ref[RS_THREADS / 32];
-    __shared__ float s_amax[RS_THREADS / 32];
-    __shared__ int s_aidx[RS_THREADS / 32];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const long long warp0 = (long long)blockIdx.x * (RS_THREADS / 32) + (threadIdx.x >> 5);
+    const long long n_warps = (long long)gridDim.x * (RS_THREADS / 32);
 
-    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+    for (long long item = warp0; item < n_items; item += n_warps) {
         const int slice_id = (int)(item % a.n_slices);
         const int dense_row = (int)(item / a.n_slices);
         const int b = dense_row / rows_per_seq;
@@ -141,7 +184,7 @@ accept_rowstats_kernel(AcceptLaunch a)
                 const float ymax = m4 * c_hi + 1.f;
                 if (ymax > ref) {   // rare: the running reference has to grow
                     const float nr = ceilf(ymax);
-                    sum = scalbn(sum, (int)fmaxf(ref - nr, -2000.f));
+                    sum = scale_down_pow2(sum, ref - nr);
                     ref = nr;
                 }
                 const float e0 = ex2_approx(fmaf(x0, c_lo, fmaf(x0, c_hi, -ref)));
@@ -156,31 +199,31 @@ accept_rowstats_kernel(AcceptLaunch a)
             // lo is a multiple of 4; the row base is 16-byte aligned
             const int n4 = (hi - lo) >> 2;
             const float *base = row + lo;
-            for (int v0 = threadIdx.x; v0 < n4; v0 += RS_THREADS * RS_UNROLL) {
+            for (int v0 = lane; v0 < n4; v0 += 32 * RS_UNROLL) {
                 float4 x[RS_UNROLL];
 #pragma unroll
                 for (int u = 0; u < RS_UNROLL; ++u) {
-                    const int v = v0 + u * RS_THREADS;
+                    const int v = v0 + u * 32;
                     x[u] = (v < n4) ? ld_stream_f4(base + 4 * (long long)v)
                                     : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F,
                                                   -CUDART_INF_F);
                 }
 #pragma unroll
                 for (int u = 0; u < RS_UNROLL; ++u) {
-                    const int v = v0 + u * RS_THREADS;
+                    const int v = v0 + u * 32;
                     if (v < n4) consume4(x[u].x, x[u].y, x[u].z, x[u].w, lo + 4 * v);
                 }
             }
             // ragged tail (vocab not a multiple of 4): at most 3 elements, last slice only
             const int tail0 = lo + 4 * n4;
-            if (threadIdx.x == 0 && tail0 < hi) {
+            if (lane == 0 && tail0 < hi) {
                 float t[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) t[u] = (tail0 + u < hi) ? row[tail0 + u] : -CUDART_INF_F;
                 consume4(t[0], t[1], t[2], t[3], tail0);
             }
         } else {
-            for (int k0 = lo + 4 * threadIdx.x; k0 < hi; k0 += 4 * RS_THREADS) {
+            for (int k0 = lo + 4 * lane; k0 < hi; k0 += 4 * 32) {
                 float t[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) t[u] = (k0 + u < hi) ? __ldg(row + k0 + u) : -CUDART_INF_F;
@@ -188,32 +231,22 @@ accept_rowstats_kernel(AcceptLaunch a)
             }
         }
 
-        // block reduction: warp shuffles, then one value per warp through shared memory
+        // warp reduction
+        if (greedy) {
 #pragma unroll
-        for (int m = 16; m > 0; m >>= 1) {
-            if (greedy) {
+            for (int m = 16; m > 0; m >>= 1) {
                 const float v2 = __shfl_xor_sync(0xffffffffu, amax, m);
                 const int i2 = __shfl_xor_sync(0xffffffffu, aidx, m);
                 merge_argmax(amax, aidx, v2, i2);
-            } else {
-                const float r2 = __shfl_xor_sync(0xffffffffu, ref, m);
-                const double s2 = shfl_xor_f64(sum, m);
-                merge_stats(ref, sum, r2, s2);
             }
+        } else {
+            float r = ref;
+#pragma unroll
+            for (int m = 16; m > 0; m >>= 1) r = fmaxf(r, __shfl_xor_sync(0xffffffffu, r, m));
+            sum = warp_sum_f64(scale_down_pow2(sum, ref - r));
+            ref = r;
         }
-        __syncthreads();   // previous item's readers are done with the shared arrays
         if (lane == 0) {
-            s_sum[warp] = sum;
-            s_ref[warp] = ref;
-            s_amax[warp] = amax;
-            s_aidx[warp] = aidx;
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            for (int w = 1; w < RS_THREADS / 32; ++w) {
-                if (greedy) merge_argmax(amax, aidx, s_amax[w], s_aidx[w]);
-                else merge_stats(ref, sum, s_ref[w], s_sum[w]);
-            }
             RowPartial out;
             out.sum = sum;
             out.ref = ref;
@@ -226,36 +259,21 @@ accept_rowstats_kernel(AcceptLaunch a)
 }
 
 // ---------------------------------------------------------------------------------------------
-// Kernel 2: decisions and sampling, one block per sequence.
+// Kernel 2: ln Z per row, ratios, first rejection.  One block per sequence.
 // ---------------------------------------------------------------------------------------------
-// four consecutive logits starting at k0 (k0 % 4 == 0), -inf past the vocabulary
-__device__ __forceinline__ void load4(const float *row, int k0, int V, bool vec, float x[4])
-{
-    if (vec && k0 + 3 < V) {
-        const float4 v = *reinterpret_cast<const float4 *>(row + k0);
-        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
-    } else {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) x[u] = (k0 + u < V) ? row[k0 + u] : -CUDART_INF_F;
-    }
-}
-
-__global__ void __launch_bounds__(FIN_THREADS)
-accept_finish_kernel(AcceptLaunch a)
+__global__ void __launch_bounds__(128)
+accept_decide_kernel(AcceptLaunch a)
 {
     const sv_accept_params &p = a.p;
-    extern __shared__ double dyn[];          // [3 * n_seg]: positive-part sums of a, of b, all of a
     __shared__ double s_logz[2 * 64 + 1];    // ln Z per dense row (natural log, of exp(x/T))
     __shared__ double s_rsum[2 * 64 + 1];    // merged sum and reference of each dense row
     __shared__ float s_rref[2 * 64 + 1];
     __shared__ int s_amax_idx[64 + 1];
-    __shared__ int s_n, s_ok;
-    __shared__ double s_red[2 * (FIN_THREADS / 32)];
     __shared__ double s_ratio[64];
     __shared__ unsigned char s_code[64];
 
     const int b = blockIdx.x;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x;
     const int gmax = p.gamma_max;
     const int rows_per_seq = 2 * gmax + 1;
     const int g = seq_gamma(p, b);
@@ -269,7 +287,7 @@ accept_finish_kernel(AcceptLaunch a)
     int32_t *out = p.out_tokens + (long long)b * (gmax + 1);
 
     // ---- merge the slice statistics of every row this sequence has
-    for (int j = tid; j < rows_per_seq; j += FIN_THREADS) {
+    for (int j = tid; j < rows_per_seq; j += blockDim.x) {
         const bool is_target = j <= gmax;
         const int i = is_target ? j : j - gmax - 1;
         const bool have = is_target ? (i <= g) : (i < g && !greedy);
@@ -293,11 +311,11 @@ accept_finish_kernel(AcceptLaunch a)
             else           { if (p.logZ_q != nullptr) p.logZ_q[p.cu_d[b] + i] = lz; }
         }
     }
-    for (int i = tid; i <= gmax; i += FIN_THREADS) out[i] = -1;
+    for (int i = tid; i <= gmax; i += blockDim.x) out[i] = -1;
     __syncthreads();
 
     // ---- ratio and decision of every draft position in parallel (float64) ...
-    for (int i = tid; i < g; i += FIN_THREADS) {
+    for (int i = tid; i < g; i += blockDim.x) {
         const int xi = x[i];
         double r = 0.0;
         int code;   // 0 reject, 1 accept, 2 non-finite partition function
@@ -342,45 +360,81 @@ accept_finish_kernel(AcceptLaunch a)
         if (!greedy && ok && !isfinite(s_logz[n])) ok = 0;
         if (!ok) set_status(p.device_status, SV_DEV_NONFINITE);
         if (flags != 0 && p.flag_count != nullptr) atomicAdd(p.flag_count, flags);
-        s_n = n;
-        s_ok = ok;
         p.n_accepted[b] = ok ? n : 0;
         if (ok) {
             for (int i = 0; i < n; ++i) out[i] = x[i];
             if (greedy) out[n] = s_amax_idx[n];
         }
+        SeqRecord rec;
+        rec.n = n;
+        rec.mode = (greedy || !ok) ? 0 : (n < g ? 1 : 2);
+        rec.ref_p = rec.ref_q = 0.f;
+        rec.sum_p_hat = rec.sum_q_hat = 1.0;
+        if (rec.mode != 0) {
+            rec.ref_p = s_rref[n];
+            rec.sum_p_hat = s_rsum[n];
+            if (rec.mode == 1) {
+                rec.ref_q = s_rref[gmax + 1 + n];
+                rec.sum_q_hat = s_rsum[gmax + 1 + n];
+            }
+        }
+        a.records[b] = rec;
     }
-    __syncthreads();
-    if (greedy || !s_ok) return;
+}
 
-    // ---- sample the next token from row n: residual max(0, p_n - q_n), or p_gamma (bonus)
-    const int n = s_n;
-    const bool residual = n < g;
-    const float *trow = t_rows + (long long)n * p.row_stride;
-    const float *drow = residual ? d_rows + (long long)n * p.row_stride : nullptr;
+// four consecutive logits starting at k0 (k0 % 4 == 0), -inf past the vocabulary
+__device__ __forceinline__ void load4(const float *row, int k0, int V, bool vec, float x[4])
+{
+    if (vec && k0 + 3 < V) {
+        const float4 v = *reinterpret_cast<const float4 *>(row + k0);
+        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    } else {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) x[u] = (k0 + u < V) ? row[k0 + u] : -CUDART_INF_F;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Kernel 3: float64 segment sums of the sampled row(s).  grid = batch * splits.
+//   a_k = 2^(t_k c - ref_p), b_k = 2^(d_k c - ref_q), c = log2(e)/T
+//   per segment: sum of a over {p_k > q_k}, sum of b over the same set, sum of all a
+//   per block: sum of all a and all b (the exact partition sums, up to 2^ref)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(SEG_THREADS)
+accept_segsum_kernel(AcceptLaunch a)
+{
+    const sv_accept_params &p = a.p;
+    __shared__ double s_red[2 * (SEG_THREADS / 32)];
+    const int b = blockIdx.x / a.splits, sp = blockIdx.x % a.splits;
+    const SeqRecord rec = a.records[b];
+    if (rec.mode == 0) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool residual = rec.mode == 1;
+    const int V = p.vocab, n_seg = a.n_seg;
+    const double c = 1.4426950408889634 / (double)seq_temperature(p, b);
+    const float *trow = p.target_logits + ((long long)p.cu_q[b] + rec.n) * p.row_stride;
+    const float *drow = residual ? p.draft_logits + ((long long)p.cu_d[b] + rec.n) * p.row_stride : nullptr;
     const bool vec = a.vec_ok != 0;
-    const int n_seg = (V + SEG - 1) / SEG;
-    double *seg_ap = dyn, *seg_bp = dyn + n_seg, *seg_a = dyn + 2 * n_seg;
-    const double c = 1.4426950408889634 / T;
-    const double ref_p = (double)s_rref[n];
-    const double ref_q = residual ? (double)s_rref[gmax + 1 + n] : 0.0;
+    const double ref_p = (double)rec.ref_p, ref_q = (double)rec.ref_q;
     // first-pass partition sums, good to ~1e-7: only used to decide the sign of p_k - q_k
-    const double inv_zp_hat = 1.0 / s_rsum[n];
-    const double inv_zq_hat = residual ? 1.0 / s_rsum[gmax + 1 + n] : 0.0;
+    const double inv_zp_hat = 1.0 / rec.sum_p_hat, inv_zq_hat = 1.0 / rec.sum_q_hat;
+    double *seg_ap = a.seg + (size_t)b * 3 * n_seg, *seg_bp = seg_ap + n_seg, *seg_a = seg_bp + n_seg;
 
+    const int per = (n_seg + a.splits - 1) / a.splits;
+    const int s_begin = sp * per, s_end = min(n_seg, s_begin + per);
     double tot_a = 0.0, tot_b = 0.0;
-    for (int s = warp; s < n_seg; s += FIN_THREADS / 32) {
+    for (int s = s_begin + warp; s < s_end; s += SEG_THREADS / 32) {
         const int k0 = s * SEG + 4 * lane;
         float xt[4], xd[4];
         load4(trow, k0, V, vec, xt);
-        double sa = 0.0, sap = 0.0, sbp = 0.0, sb = 0.0;
         if (residual) load4(drow, k0, V, vec, xd);
+        double sa = 0.0, sap = 0.0, sbp = 0.0, sb = 0.0;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const double ak = exp2((double)xt[u] * c - ref_p);
+            const double ak = exp2_f64((double)xt[u] * c - ref_p);
             sa += ak;
             if (residual) {
-                const double bk = exp2((double)xd[u] * c - ref_q);
+                const double bk = exp2_f64((double)xd[u] * c - ref_q);
                 sb += bk;
                 if (ak * inv_zp_hat > bk * inv_zq_hat) { sap += ak; sbp += bk; }
             }
@@ -393,24 +447,52 @@ accept_finish_kernel(AcceptLaunch a)
     }
     tot_a = warp_sum_f64(tot_a);
     tot_b = warp_sum_f64(tot_b);
-    if (lane == 0) { s_red[warp] = tot_a; s_red[FIN_THREADS / 32 + warp] = tot_b; }
+    if (lane == 0) { s_red[warp] = tot_a; s_red[SEG_THREADS / 32 + warp] = tot_b; }
     __syncthreads();
-    if (warp != 0) return;   // the rest is one warp's work
+    if (tid == 0) {
+        double za = 0.0, zb = 0.0;
+        for (int w = 0; w < SEG_THREADS / 32; ++w) { za += s_red[w]; zb += s_red[SEG_THREADS / 32 + w]; }
+        a.totals[((size_t)b * MAX_SPLITS + sp) * 2] = za;
+        a.totals[((size_t)b * MAX_SPLITS + sp) * 2 + 1] = zb;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Kernel 4: inverse CDF.  One warp per sequence.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32)
+accept_pick_kernel(AcceptLaunch a)
+{
+    const sv_accept_params &p = a.p;
+    const int b = blockIdx.x, lane = threadIdx.x;
+    const SeqRecord rec = a.records[b];
+    if (rec.mode == 0) return;
+    const bool residual = rec.mode == 1;
+    const int V = p.vocab, n_seg = a.n_seg, n = rec.n;
+    const double c = 1.4426950408889634 / (double)seq_temperature(p, b);
+    const float *trow = p.target_logits + ((long long)p.cu_q[b] + n) * p.row_stride;
+    const float *drow = residual ? p.draft_logits + ((long long)p.cu_d[b] + n) * p.row_stride : nullptr;
+    const bool vec = a.vec_ok != 0;
+    const double ref_p = (double)rec.ref_p, ref_q = (double)rec.ref_q;
+    const double *seg_ap = a.seg + (size_t)b * 3 * n_seg, *seg_bp = seg_ap + n_seg, *seg_a = seg_bp + n_seg;
 
     double Zp = 0.0, Zq = 0.0;
-    for (int w = 0; w < FIN_THREADS / 32; ++w) { Zp += s_red[w]; Zq += s_red[FIN_THREADS / 32 + w]; }
+    for (int sp = 0; sp < a.splits; ++sp) {
+        Zp += a.totals[((size_t)b * MAX_SPLITS + sp) * 2];
+        Zq += a.totals[((size_t)b * MAX_SPLITS + sp) * 2 + 1];
+    }
     const double inv_zp = 1.0 / Zp, inv_zq = residual ? 1.0 / Zq : 0.0;
 
     // total mass; lane l owns the contiguous segments [l*per, (l+1)*per)
     const int per = (n_seg + 31) / 32;
     const int s_lo = min(lane * per, n_seg), s_hi = min(s_lo + per, n_seg);
-    auto seg_w = [&](int s, bool use_resid) {
-        return use_resid ? seg_ap[s] * inv_zp - seg_bp[s] * inv_zq : seg_a[s] * inv_zp;
+    auto seg_w = [&](int s, bool use_r) {
+        return use_r ? seg_ap[s] * inv_zp - seg_bp[s] * inv_zq : seg_a[s] * inv_zp;
     };
     double mine = 0.0;
     if (residual) for (int s = s_lo; s < s_hi; ++s) mine += seg_w(s, true);
     double W = warp_sum_f64(mine);
-    bool use_resid = residual && (W > 0.0);     // no residual mass: fall back to p_n
+    const bool use_resid = residual && (W > 0.0);     // no residual mass: fall back to p_n
     if (!use_resid) {
         mine = 0.0;
         for (int s = s_lo; s < s_hi; ++s) mine += seg_w(s, false);
@@ -434,7 +516,6 @@ accept_finish_kernel(AcceptLaunch a)
         if (seg_found == n_seg && cum + w > target) { seg_found = s; seg_base = cum; }
         cum += w;
     }
-    // lowest segment over the warp
     int best = seg_found;
 #pragma unroll
     for (int m = 16; m > 0; m >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, m));
@@ -442,25 +523,29 @@ accept_finish_kernel(AcceptLaunch a)
     double base = 0.0;
     if (who != 0) base = shfl_idx_f64(seg_base, __ffs(who) - 1);
 
-    // resolve inside the segment with exact float64 weights; if rounding pushed the target
-    // past this segment, walk on; if nothing qualifies, take the last positive weight.
+    // exact float64 weights of four consecutive tokens
+    auto weights4 = [&](int k0, double w[4]) {
+        float xt[4], xd[4];
+        load4(trow, k0, V, vec, xt);
+        if (use_resid) load4(drow, k0, V, vec, xd);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const double pk = exp2_f64((double)xt[u] * c - ref_p) * inv_zp;
+            w[u] = use_resid ? fmax(pk - exp2_f64((double)xd[u] * c - ref_q) * inv_zq, 0.0) : pk;
+        }
+    };
+
+    // resolve inside the segment; if rounding pushed the target past it, walk on; if nothing
+    // qualifies, take the last positive weight.
     int y = -1, last_pos = -1;
     int s = best;
     if (best >= n_seg) { s = 0; base = 0.0; }    // target at or beyond the total: walk everything
     for (; s < n_seg && y < 0; ++s) {
         const int k0 = s * SEG + 4 * lane;
-        float xt[4], xd[4];
-        load4(trow, k0, V, vec, xt);
-        if (use_resid) load4(drow, k0, V, vec, xd);
         double w[4], loc = 0.0;
+        weights4(k0, w);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const double pk = exp2((double)xt[u] * c - ref_p) * inv_zp;
-            double wk = pk;
-            if (use_resid) wk = fmax(pk - exp2((double)xd[u] * c - ref_q) * inv_zq, 0.0);
-            w[u] = wk;
-            loc += wk;
-        }
+        for (int u = 0; u < 4; ++u) loc += w[u];
         double inc = loc;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
@@ -485,50 +570,55 @@ accept_finish_kernel(AcceptLaunch a)
     }
     if (y < 0) {
         // target at or beyond the total mass: last token with positive weight
-        if (last_pos < 0) {
-            for (int s2 = n_seg - 1; s2 >= 0 && last_pos < 0; --s2) {
-                const int k0 = s2 * SEG + 4 * lane;
-                float xt[4], xd[4];
-                load4(trow, k0, V, vec, xt);
-                if (use_resid) load4(drow, k0, V, vec, xd);
-                int lp = -1;
+        for (int s2 = n_seg - 1; s2 >= 0 && last_pos < 0; --s2) {
+            const int k0 = s2 * SEG + 4 * lane;
+            double w[4];
+            weights4(k0, w);
+            int lp = -1;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const double pk = exp2((double)xt[u] * c - ref_p) * inv_zp;
-                    double wk = pk;
-                    if (use_resid) wk = fmax(pk - exp2((double)xd[u] * c - ref_q) * inv_zq, 0.0);
-                    if (wk > 0.0) lp = k0 + u;
-                }
-                const unsigned pos = __ballot_sync(0xffffffffu, lp >= 0);
-                if (pos != 0) last_pos = __shfl_sync(0xffffffffu, lp, 31 - __clz(pos));
-            }
+            for (int u = 0; u < 4; ++u)
+                if (w[u] > 0.0) lp = k0 + u;
+            const unsigned pos = __ballot_sync(0xffffffffu, lp >= 0);
+            if (pos != 0) last_pos = __shfl_sync(0xffffffffu, lp, 31 - __clz(pos));
         }
         y = last_pos;
     }
-    if (lane == 0) out[n] = y;
+    if (lane == 0) p.out_tokens[(long long)b * (p.gamma_max + 1) + n] = y;
 }
 
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
 static int pick_slice(const sv_accept_params *p)
 {
-    // aim for at least ~4 blocks per SM worth of (row, slice) items, slices of 2K..16K elements
+    // one warp per (row, slice): aim for a few items per resident warp, slices of 2K..16K elements
     const long long rows = (long long)p->batch * (2 * p->gamma_max + 1);
-    const long long want = 4LL * sm_count();
-    int slice = 16384;
+    const long long want = 4LL * sm_count() * 40;
+    int slice = MAX_SLICE;
     while (slice > MIN_SLICE && rows * ((p->vocab + slice - 1) / slice) < want) slice >>= 1;
     return slice;
 }
 
-}  // namespace sv
+static size_t align256(size_t n) { return (n + 255) & ~(size_t)255; }
 
-extern "C" size_t spec_accept_sample_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t vocab)
+struct AcceptLayout {
+    size_t partials, records, seg, totals, total;
+};
+
+static AcceptLayout accept_layout(int batch, int gamma_max, int vocab, int slice)
 {
-    if (batch <= 0 || gamma_max < 0 || vocab <= 0) return 0;
-    const size_t n_slices = ((size_t)vocab + sv::MIN_SLICE - 1) / sv::MIN_SLICE;
-    return (size_t)batch * (2 * (size_t)gamma_max + 1) * n_slices * sizeof(sv::RowPartial);
+    AcceptLayout l;
+    const size_t n_slices = ((size_t)vocab + slice - 1) / slice;
+    const size_t n_seg = ((size_t)vocab + SEG - 1) / SEG;
+    l.partials = 0;
+    l.records = align256((size_t)batch * (2 * (size_t)gamma_max + 1) * n_slices * sizeof(RowPartial));
+    l.seg = l.records + align256((size_t)batch * sizeof(SeqRecord));
+    l.totals = l.seg + align256((size_t)batch * 3 * n_seg * sizeof(double));
+    l.total = l.totals + align256((size_t)batch * MAX_SPLITS * 2 * sizeof(double));
+    return l;
 }
 
-extern "C" sv_status spec_accept_sample(const sv_accept_params *p, void *workspace,
-                                        size_t workspace_bytes, void *stream)
+static sv_status check_accept(const sv_accept_params *p)
 {
     if (p == nullptr || p->batch <= 0 || p->vocab <= 0 || p->gamma_max < 0) return SV_EINVAL;
     if (p->gamma_max > 64) return SV_EUNSUPPORTED;
@@ -541,37 +631,76 @@ extern "C" sv_status spec_accept_sample(const sv_accept_params *p, void *workspa
     if (p->gamma_max > 0 && p->draft_tokens == nullptr) return SV_EINVAL;
     if (p->row_stride < p->vocab) return SV_EINVAL;
     if (!(p->temperature >= 0.f)) return SV_EINVAL;
+    return SV_OK;
+}
+
+// the four launches; `scratch` holds accept_layout(..., slice).total bytes
+static sv_status launch_accept(const sv_accept_params *p, void *scratch, int slice, cudaStream_t stream)
+{
+    const AcceptLayout l = accept_layout(p->batch, p->gamma_max, p->vocab, slice);
+    uint8_t *base = static_cast<uint8_t *>(scratch);
+    AcceptLaunch a;
+    a.p = *p;
+    a.partials = reinterpret_cast<RowPartial *>(base + l.partials);
+    a.records = reinterpret_cast<SeqRecord *>(base + l.records);
+    a.seg = reinterpret_cast<double *>(base + l.seg);
+    a.totals = reinterpret_cast<double *>(base + l.totals);
+    a.slice = slice;
+    a.n_slices = (p->vocab + slice - 1) / slice;
+    a.n_seg = (p->vocab + SEG - 1) / SEG;
+    a.vec_ok = (p->row_stride % 4 == 0) && aligned16(p->target_logits) &&
+               (p->draft_logits == nullptr || aligned16(p->draft_logits));
+    // blocks per sequence in the float64 pass: enough to occupy the machine, at least 8 segments each
+    int splits = (4 * sm_count() + p->batch - 1) / p->batch;
+    if (splits > MAX_SPLITS) splits = MAX_SPLITS;
+    if (splits > (a.n_seg + 7) / 8) splits = (a.n_seg + 7) / 8;
+    if (splits < 1) splits = 1;
+    a.splits = splits;
+
+    const long long n_items = (long long)p->batch * (2 * p->gamma_max + 1) * a.n_slices;
+    const long long blocks_needed = (n_items + RS_THREADS / 32 - 1) / (RS_THREADS / 32);
+    static int blocks_per_sm = 0;       // resident blocks per SM, asked once
+    if (blocks_per_sm == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, accept_rowstats_kernel, RS_THREADS, 0) !=
+                cudaSuccess || n < 1)
+            n = 2;
+        blocks_per_sm = n;
+    }
+    const long long cap = (long long)blocks_per_sm * sm_count();
+    accept_rowstats_kernel<<<(int)(blocks_needed < cap ? blocks_needed : cap), RS_THREADS, 0, stream>>>(a);
+    sv_status st = launch_check();
+    if (st != SV_OK) return st;
+    accept_decide_kernel<<<p->batch, 128, 0, stream>>>(a);
+    st = launch_check();
+    if (st != SV_OK) return st;
+    const bool any_sampling = p->temperature_per_seq != nullptr || p->temperature > 0.f;
+    if (!any_sampling) return SV_OK;
+    accept_segsum_kernel<<<(unsigned)(splits * p->batch), SEG_THREADS, 0, stream>>>(a);
+    st = launch_check();
+    if (st != SV_OK) return st;
+    accept_pick_kernel<<<p->batch, 32, 0, stream>>>(a);
+    return launch_check();
+}
+
+}  // namespace sv
+
+extern "C" size_t spec_accept_sample_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t vocab)
+{
+    if (batch <= 0 || gamma_max < 0 || vocab <= 0) return 0;
+    return sv::accept_layout(batch, gamma_max, vocab, sv::MIN_SLICE).total;
+}
+
+extern "C" sv_status spec_accept_sample(const sv_accept_params *p, void *workspace,
+                                        size_t workspace_bytes, void *stream)
+{
+    sv_status st = sv::check_accept(p);
+    if (st != SV_OK) return st;
     if (workspace == nullptr ||
         workspace_bytes < spec_accept_sample_workspace_bytes(p->batch, p->gamma_max, p->vocab))
         return SV_EWORKSPACE;
     if (!sv::aligned16(workspace)) return SV_EALIGN;
-
-    const int n_seg = (p->vocab + sv::SEG - 1) / sv::SEG;
-    const size_t dyn = 3 * sizeof(double) * (size_t)n_seg;
-    if (dyn > 200 * 1024) return SV_EUNSUPPORTED;
-
-    sv::AcceptLaunch a;
-    a.p = *p;
-    a.partials = static_cast<sv::RowPartial *>(workspace);
-    a.slice = sv::pick_slice(p);
-    a.n_slices = (p->vocab + a.slice - 1) / a.slice;
-    a.vec_ok = (p->row_stride % 4 == 0) && sv::aligned16(p->target_logits) &&
-               (p->draft_logits == nullptr || sv::aligned16(p->draft_logits));
-
-    const long long n_items = (long long)p->batch * (2 * p->gamma_max + 1) * a.n_slices;
-    const long long cap = 8LL * sv::sm_count();
-    const int grid = (int)(n_items < cap ? n_items : cap);
-    sv::accept_rowstats_kernel<<<grid, sv::RS_THREADS, 0, (cudaStream_t)stream>>>(a);
-    sv_status st = sv::launch_check();
-    if (st != SV_OK) return st;
-
-    if (dyn > 48 * 1024) {
-        if (cudaFuncSetAttribute(sv::accept_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)dyn) != cudaSuccess)
-            return SV_ECUDA;
-    }
-    sv::accept_finish_kernel<<<p->batch, sv::FIN_THREADS, dyn, (cudaStream_t)stream>>>(a);
-    return sv::launch_check();
+    return sv::launch_accept(p, workspace, sv::pick_slice(p), (cudaStream_t)stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -579,9 +708,9 @@ extern "C" sv_status spec_accept_sample(const sv_accept_params *p, void *workspa
 // ---------------------------------------------------------------------------------------------
 namespace sv {
 
-// Slice statistics of one call live here instead of in a caller's workspace.  The array is part
-// of the library image: every GPU that loads the library holds these bytes until the process
-// exits.  All calls on a device share it.
+// The intermediate results of one call live here instead of in a caller's workspace.  The array
+// is part of the library image: every GPU that loads the library holds these bytes until the
+// process exits.  All calls on a device share it.
 static __device__ __align__(256) unsigned char g_accept_static_scratch[SV_ACCEPT_STATIC_SCRATCH_BYTES];
 
 constexpr int MAX_DEVICES = 64;
@@ -591,31 +720,12 @@ static void *g_static_scratch_ptr[MAX_DEVICES];   // device address of the array
 
 extern "C" sv_status spec_accept_sample_static(const sv_accept_params *p, void *stream)
 {
-    if (p == nullptr || p->batch <= 0 || p->vocab <= 0 || p->gamma_max < 0) return SV_EINVAL;
-    if (p->gamma_max > 64) return SV_EUNSUPPORTED;
-    if (p->target_logits == nullptr || p->gamma == nullptr || p->cu_q == nullptr ||
-        p->cu_d == nullptr || p->n_accepted == nullptr || p->out_tokens == nullptr)
-        return SV_EINVAL;
-    const bool any_sampling = p->temperature_per_seq != nullptr || p->temperature > 0.f;
-    if (any_sampling && (p->draft_logits == nullptr || p->u_accept == nullptr || p->u_sample == nullptr))
-        return SV_EINVAL;
-    if (p->gamma_max > 0 && p->draft_tokens == nullptr) return SV_EINVAL;
-    if (p->row_stride < p->vocab) return SV_EINVAL;
-    if (!(p->temperature >= 0.f)) return SV_EINVAL;
-    const int n_seg = (p->vocab + sv::SEG - 1) / sv::SEG;
-    const size_t dyn = 3 * sizeof(double) * (size_t)n_seg;
-    if (dyn > 200 * 1024) return SV_EUNSUPPORTED;
-
-    sv::AcceptLaunch a;
-    a.p = *p;
-    a.slice = sv::pick_slice(p);
-    a.n_slices = (p->vocab + a.slice - 1) / a.slice;
-    a.vec_ok = (p->row_stride % 4 == 0) && sv::aligned16(p->target_logits) &&
-               (p->draft_logits == nullptr || sv::aligned16(p->draft_logits));
-    const unsigned long long n_items =
-        (unsigned long long)p->batch * (2ull * p->gamma_max + 1) * (unsigned long long)a.n_slices;
-    // the problem must fit the built-in array: one 32-byte record per (row, slice)
-    if (n_items * sizeof(sv::RowPartial) > (unsigned long long)SV_ACCEPT_STATIC_SCRATCH_BYTES)
+    sv_status st = sv::check_accept(p);
+    if (st != SV_OK) return st;
+    // the problem must fit the built-in array
+    const int slice = sv::pick_slice(p);
+    if (sv::accept_layout(p->batch, p->gamma_max, p->vocab, slice).total >
+        (size_t)SV_ACCEPT_STATIC_SCRATCH_BYTES)
         return SV_EWORKSPACE;
 
     // In host code the array's name is only a handle; its device address has to be asked for,
@@ -628,18 +738,5 @@ extern "C" sv_status spec_accept_sample_static(const sv_accept_params *p, void *
             return SV_ECUDA;
         sv::g_static_scratch_ptr[dev] = ptr;
     }
-    a.partials = static_cast<sv::RowPartial *>(sv::g_static_scratch_ptr[dev]);
-
-    const long long cap = 8LL * sv::sm_count();
-    const int grid = (int)((long long)n_items < cap ? (long long)n_items : cap);
-    sv::accept_rowstats_kernel<<<grid, sv::RS_THREADS, 0, (cudaStream_t)stream>>>(a);
-    sv_status st = sv::launch_check();
-    if (st != SV_OK) return st;
-    if (dyn > 48 * 1024) {
-        if (cudaFuncSetAttribute(sv::accept_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)dyn) != cudaSuccess)
-            return SV_ECUDA;
-    }
-    sv::accept_finish_kernel<<<p->batch, sv::FIN_THREADS, dyn, (cudaStream_t)stream>>>(a);
-    return sv::launch_check();
+    return sv::launch_accept(p, sv::g_static_scratch_ptr[dev], slice, (cudaStream_t)stream);
 }

@@ -86,7 +86,7 @@ def test_two_calls_in_a_row_match_the_regular_entry_point():
 
 
 def test_problem_larger_than_the_built_in_array_is_refused():
-    B, gmax, V = 4096, 16, 128256            # 4096 * 33 * 8 slices * 32 B = 34.6 MB > 4 MiB
+    B, gmax, V = 4096, 16, 128256            # slice statistics alone: 4096 * 33 * 8 * 32 B = 34.6 MB > 8 MiB
     z = torch.zeros(1, dtype=torch.float32, device=DEV)
     i = torch.zeros(1, dtype=torch.int32, device=DEV)
     p = sv.AcceptParams()
