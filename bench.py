@@ -45,8 +45,10 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
 
 
-def workload_inputs(cfg, rank, batch=None, gamma=None):
+def workload_inputs(cfg, rank, batch=None, gamma=None, gamma_max=None):
     cfg = synth.scaled(cfg, seed=cfg.seed + 1000 * rank)
+    if gamma_max is not None:
+        cfg = synth.scaled(cfg, gamma_max=gamma_max)
     if gamma is not None:
         cfg = synth.scaled(cfg, gamma_lo=gamma, gamma_hi=gamma)
     if batch:
@@ -91,7 +93,7 @@ def run_reference(args):
         return
     import oracle
     oracle.build()
-    cfg, seq_len, gamma, cu_q, cu_d = workload_inputs(synth.CONFIGS[args.workload], 0, args.batch, args.gamma)
+    cfg, seq_len, gamma, cu_q, cu_d = workload_inputs(synth.CONFIGS[args.workload], 0, args.batch, args.gamma, args.gamma_max)
     n_seq = min(args.oracle_seqs or 4, cfg.batch)
     sub, kv, q, li = sample_inputs(cfg, seq_len, gamma, cu_q, cu_d, n_seq)
     times, toks = [], 0
@@ -189,7 +191,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(DEV))
 
     base_cfg = synth.CONFIGS[args.workload]
-    cfg, seq_len, gamma, cu_q, cu_d = workload_inputs(base_cfg, rank, args.batch, args.gamma)
+    cfg, seq_len, gamma, cu_q, cu_d = workload_inputs(base_cfg, rank, args.batch, args.gamma, args.gamma_max)
     B, gmax = cfg.batch, cfg.gamma_max
     n_q, n_d = int(cu_q[-1]), int(cu_d[-1])
     kv = synth.make_kv(cfg, seq_len, reserve_tokens=2 * (gmax + 1))
@@ -388,6 +390,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gamma", type=int, default=None,
                     help="draft length of every sequence (default: the workload's own range)")
+    ap.add_argument("--gamma-max", type=int, default=None, help="override the controller's upper bound")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the workload's batch (smaller cases for profiler captures)")
     args = ap.parse_args()

@@ -28,10 +28,10 @@
 
 namespace sv {
 
-constexpr int TILE = 128;               // tokens per tile
-constexpr int PAGES_PER_TILE = 8;
 constexpr int HD = 128;                 // head_dim of this kernel
-constexpr int SLOT_BYTES = TILE * HD * 2;          // 32 KB: one K or one V tile
+// Tokens per key tile are a template parameter: 64 (4 pages, 16 KB per K or V tile) when one
+// row group suffices -- two thread blocks then share an SM and hide each other's hand-off
+// latencies -- and 128 (8 pages, 32 KB) with two row groups, one block per SM.
 constexpr int QGROUP_BYTES = 128 * HD * 2;         // 32 KB: 128 query rows
 constexpr int MAX_BATCH_TC = 1 << 20;
 constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2 s: far beyond any legitimate wait
@@ -164,15 +164,15 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     d |= (uint64_t)2 << 61;      // 128-byte swizzle
     return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128.
-__device__ __forceinline__ uint32_t instr_desc(bool b_n_major)
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc(bool b_n_major, int n)
 {
     uint32_t d = 0;
     d |= 1u << 4;                 // accumulator fp32
     d |= 1u << 7;                 // A bf16
     d |= 1u << 10;                // B bf16
     d |= (b_n_major ? 1u : 0u) << 16;
-    d |= (uint32_t)(128 >> 3) << 17;
+    d |= (uint32_t)(n >> 3) << 17;
     d |= (uint32_t)(128 >> 4) << 24;
     return d;
 }
@@ -227,7 +227,7 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, Shar
 }
 
 // Tiles and validated gamma of one sequence; sequences with inconsistent lengths own no tiles.
-__device__ __forceinline__ int seq_tiles(const sv_attn_params &p, int b, int *gam_out, bool report)
+__device__ __forceinline__ int seq_tiles(const sv_attn_params &p, int b, int *gam_out, bool report, int tile)
 {
     int g = p.gamma[b];
     if (g < 0 || g > p.gamma_max) {
@@ -235,7 +235,7 @@ __device__ __forceinline__ int seq_tiles(const sv_attn_params &p, int b, int *ga
         g = min(max(g, 0), p.gamma_max);
     }
     const int L = p.seq_len[b];
-    int nt = (L + TILE - 1) / TILE;
+    int nt = (L + tile - 1) / tile;
     if (L < g + 1 || (long long)(L + 15) / 16 > p.block_table_stride || L > p.max_seq_len) {
         if (report) set_status(p.device_status, SV_DEV_BAD_LEN);
         nt = 0;
@@ -247,10 +247,12 @@ __device__ __forceinline__ int seq_tiles(const sv_attn_params &p, int b, int *ga
 // Walks the (sequence, kv head, tile) triples of a block's share.
 struct TileCursor {
     int b, g, t, n_tiles, gam;    // current pair, tile inside it, its tile count and gamma
-    __device__ void seek(const sv_attn_params &p, const Shared *sh, long long tile)
+    int tile_tokens;
+    __device__ void seek(const sv_attn_params &p, const Shared *sh, long long tile, int tokens)
     {
+        tile_tokens = tokens;
         b = sh->start_b;
-        n_tiles = seq_tiles(p, b, &gam, false);
+        n_tiles = seq_tiles(p, b, &gam, false, tile_tokens);
         const long long rel = tile - (long long)sh->start_prefix * p.hkv;
         g = (int)(rel / n_tiles);
         t = (int)(rel % n_tiles);
@@ -261,21 +263,29 @@ struct TileCursor {
         if (++g == p.hkv) {
             g = 0;
             n_tiles = 0;
-            while (n_tiles == 0 && ++b < p.batch) n_tiles = seq_tiles(p, b, &gam, false);
+            while (n_tiles == 0 && ++b < p.batch) n_tiles = seq_tiles(p, b, &gam, false, tile_tokens);
             if (b >= p.batch) n_tiles = 1;      // past the end: never used
         }
     }
 };
 
 // ---------------------------------------------------------------------------- main kernel
-template <int NQ>
-__global__ void __launch_bounds__(128 + 128 * NQ, 1)
+template <int NQ, int TILE>
+__global__ void __launch_bounds__(128 + 128 * NQ, (NQ == 1 && TILE == 64) ? 2 : 1)
 attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                const __grid_constant__ CUtensorMap v_map)
 {
+    constexpr int PAGES_PER_TILE = TILE / 16;
+    constexpr int SLOT_BYTES = TILE * HD * 2;          // one K or one V tile
+    constexpr int O_COL0 = 2 * TILE;                   // TMEM: two S buffers of TILE columns, then O
+    constexpr uint32_t TMEM_COLS = (2 * TILE + 128 * NQ <= 256) ? 256u : 512u;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    // carve: [Q groups][ring slots][Shared]; the dynamic window is aligned to 1024 by the launch
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // carve: [Q groups][ring slots][Shared]; the swizzled tiles need a 1024-byte aligned base
+    uint8_t *smem = smem_raw;
+    if ((smem_u32(smem) & 1023u) != 0) {               // never seen; refuse rather than compute garbage
+        if (threadIdx.x == 0) set_status(a.p.device_status, SV_DEV_TIMEOUT);
+        return;
+    }
     uint8_t *q_smem = smem;
     uint8_t *ring = smem + NQ * QGROUP_BYTES;
     Shared *sh = reinterpret_cast<Shared *>(ring + a.n_slots * SLOT_BYTES);
@@ -307,7 +317,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
         if (blockIdx.x == 0 && lane == 0) a.ws_prefix[0] = 0;
         for (int base = 0; base < batch; base += 32) {
             const int b = base + lane;
-            int v = (b < batch) ? seq_tiles(p, b, nullptr, blockIdx.x == 0) : 0;
+            int v = (b < batch) ? seq_tiles(p, b, nullptr, blockIdx.x == 0, TILE) : 0;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
                 const int t = __shfl_up_sync(0xffffffffu, v, d);
@@ -329,7 +339,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
         carry = 0;
         for (int base = 0; base < batch; base += 32) {
             const int b = base + lane;
-            const int nt = (b < batch) ? seq_tiles(p, b, nullptr, false) : 0;
+            const int nt = (b < batch) ? seq_tiles(p, b, nullptr, false, TILE) : 0;
             int v = nt;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
@@ -347,7 +357,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                          smem_u32(&sh->tmem_base)),
-                     "r"(512u)
+                     "r"(TMEM_COLS)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -369,7 +379,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
         if (t_end > t_begin && warp == 0) {
             // ================================================================ TMA producer
             TileCursor cur;
-            cur.seek(p, sh, t_begin);
+            cur.seek(p, sh, t_begin, TILE);
             uint32_t item = 0;     // ring items: 2*tile = K, 2*tile+1 = V
             for (long long tg = t_begin; tg < t_end; ++tg) {
                 const int b = cur.b;
@@ -377,7 +387,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 const int n_pages = (L + 15) >> 4;
                 const int32_t *bt = p.block_table + (long long)b * p.block_table_stride;
                 // lane l fetches (page l/2, dims half l%2) of K, then of V
-                const int page_in_tile = (lane & 15) >> 1, half = lane & 1;
+                const int page_in_tile = (lane >> 1) % PAGES_PER_TILE, half = lane & 1;
                 const int lp = cur.t * PAGES_PER_TILE + page_in_tile;
                 int phys = (int)a.n_pool_pages;       // out of range: TMA fills zeros, no traffic
                 if (lp < n_pages) {
@@ -396,7 +406,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     if (!ok) break;
                     if (lane == 0) mbar_expect_tx(full, SLOT_BYTES);
                     __syncwarp();
-                    if (lane < 16) {
+                    if (lane < 2 * PAGES_PER_TILE) {
                         const uint32_t dst = smem_u32(ring + slot * SLOT_BYTES + half * (SLOT_BYTES / 2) +
                                                       page_in_tile * 2048);
                         tma_load_4d(dst, kv == 0 ? &k_map : &v_map, half * 64, 0, cur.g, phys, full);
@@ -409,9 +419,9 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
         } else if (t_end > t_begin && warp == 1) {
             // ================================================================ MMA issuer
             if (lane == 0) {
-                const uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
+                const uint32_t idesc_qk = instr_desc(false, TILE), idesc_pv = instr_desc(true, HD);
                 TileCursor cur;
-                cur.seek(p, sh, t_begin);
+                cur.seek(p, sh, t_begin, TILE);
                 uint32_t tile_no = 0;      // tiles of this block so far (ring position)
                 uint32_t ug = 0;           // global unit counter: unit = (tile, row group)
                 uint32_t seg_no = 0;
@@ -435,11 +445,12 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                         if (!ok) return;
                         const uint32_t ka = smem_u32(ring + slot * SLOT_BYTES);
                         const uint32_t qa = smem_u32(q_smem + q * QGROUP_BYTES);
-                        const uint32_t d = tmem + ((ug + u) & 1) * 128;
+                        const uint32_t d = tmem + ((ug + u) & 1) * TILE;
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {
-                            const uint32_t off = (ks >> 2) * (SLOT_BYTES / 2) + (ks & 3) * 32;
-                            tc_mma_ss(d, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024),
+                            const uint32_t koff = (ks >> 2) * (SLOT_BYTES / 2) + (ks & 3) * 32;
+                            const uint32_t qoff = (ks >> 2) * (QGROUP_BYTES / 2) + (ks & 3) * 32;
+                            tc_mma_ss(d, smem_desc(qa + qoff, 16, 1024), smem_desc(ka + koff, 16, 1024),
                                       idesc_qk, ks > 0);
                         }
                         tc_commit(smem_u32(&sh->s_full[(ug + u) & 1]));
@@ -459,10 +470,10 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                         if (!ok) break;
                         tc_fence_after();
                         const uint32_t va = smem_u32(ring + slot * SLOT_BYTES);
-                        const uint32_t pa = tmem + (gu & 1) * 128;       // P overlays S, 64 columns
-                        const uint32_t d = tmem + 256 + q * 128;
+                        const uint32_t pa = tmem + (gu & 1) * TILE;      // P overlays S, TILE/2 columns
+                        const uint32_t d = tmem + O_COL0 + q * 128;
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)
+                        for (int ks = 0; ks < TILE / 16; ++ks)
                             tc_mma_ts(d, pa + ks * 8, smem_desc(va + ks * 2048, SLOT_BYTES / 2, 1024),
                                       idesc_pv, (ti > 0 || ks > 0) ? 1u : 0u);
                         tc_commit(smem_u32(&sh->o_done[q]));
@@ -488,7 +499,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
             const int r = q * 128 + r_in;                      // row of the (b, g) pair
             const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
             TileCursor cur;
-            cur.seek(p, sh, t_begin);
+            cur.seek(p, sh, t_begin, TILE);
             uint32_t ug = 0, kq = 0;       // global unit counter, units of this group so far
             uint32_t seg_no = 0;
             bool ok = true;
@@ -535,10 +546,10 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     continue;
                 }
                 float m_ref = -CUDART_INF_F, l_sum = 0.f;
-                const uint32_t o_addr = tmem + lane_addr + 256 + q * 128;
+                const uint32_t o_addr = tmem + lane_addr + O_COL0 + q * 128;
                 for (int ti = 0; ti < seg_tiles && ok; ++ti) {
                     const uint32_t gu = ug + ti * nq_seg + q;
-                    const uint32_t s_addr = tmem + lane_addr + (gu & 1) * 128;
+                    const uint32_t s_addr = tmem + lane_addr + (gu & 1) * TILE;
                     ok = bounded_wait(smem_u32(&sh->s_full[gu & 1]), (gu >> 1) & 1, sh, p.device_status);
                     if (!ok) break;
                     if (!warp_active) {                         // all 32 rows are padding
@@ -550,18 +561,18 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     const int tok0 = (cur.t + ti) * TILE;
                     const bool need_mask = tok0 + TILE - 1 > L - R;    // some row cannot see the whole tile
                     // the row's 128 scores: four loads in flight, one wait
-                    uint32_t s[128];
+                    uint32_t s[TILE];
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) tc_ld32_nowait(s_addr + ch * 32, s + ch * 32);
+                    for (int ch = 0; ch < TILE / 32; ++ch) tc_ld32_nowait(s_addr + ch * 32, s + ch * 32);
                     tc_wait_ld();
                     if (need_mask) {
 #pragma unroll
-                        for (int c = 0; c < 128; ++c)
+                        for (int c = 0; c < TILE; ++c)
                             if (tok0 + c > pos) s[c] = 0xff800000u;     // -inf
                     }
                     float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
 #pragma unroll
-                    for (int c = 0; c < 128; c += 4) {
+                    for (int c = 0; c < TILE; c += 4) {
                         m0 = fmaxf(m0, __uint_as_float(s[c]));
                         m1 = fmaxf(m1, __uint_as_float(s[c + 1]));
                         m2 = fmaxf(m2, __uint_as_float(s[c + 2]));
@@ -600,7 +611,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     // P = 2^(s*c - m_ref) as bf16 pairs, written over S (masked scores are -inf -> 0)
                     float tile_sum = 0.f;
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
+                    for (int ch = 0; ch < TILE / 32; ++ch) {
                         float sum0 = 0.f, sum1 = 0.f;
                         uint32_t pk[16];
 #pragma unroll
@@ -693,7 +704,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
     }
 }
 
@@ -776,6 +787,9 @@ bool attn_tc_supported(const sv_attn_params &p)
 
 static size_t prefix_bytes(int batch) { return (((size_t)batch + 2) * sizeof(int32_t) + 255) & ~(size_t)255; }
 
+// blocks of the main kernel: two per SM with one row group (64-token tiles), else one per SM
+static int attn_grid(int nq) { return nq == 1 ? 2 * sm_count() : sm_count(); }
+
 size_t attn_tc_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t hq, int32_t hkv,
                                int32_t head_dim, int32_t max_seq_len)
 {
@@ -784,7 +798,26 @@ size_t attn_tc_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t hq, int
     const int rows = (hq / hkv) * (gamma_max + 1);
     const int nq = (rows + 127) / 128;
     if (nq < 1 || nq > 2 || batch > MAX_BATCH_TC) return 0;
-    return prefix_bytes(batch) + (size_t)sm_count() * 2 * part_slot_floats(nq) * sizeof(float);
+    return prefix_bytes(batch) + (size_t)attn_grid(nq) * 2 * part_slot_floats(nq) * sizeof(float);
+}
+
+template <int NQ, int TILE>
+static sv_status launch_main(AttnTcLaunch &a, const sv_attn_params &p, int grid, cudaStream_t stream)
+{
+    constexpr int slot_bytes = TILE * HD * 2;
+    // shared memory an SM can give to its resident blocks (1 KB per block is reserved)
+    constexpr int blocks_per_sm = (NQ == 1 && TILE == 64) ? 2 : 1;
+    const size_t budget = (228 * 1024) / blocks_per_sm - 1024;
+    const size_t fixed = (size_t)NQ * QGROUP_BYTES + ((sizeof(Shared) + 127) & ~(size_t)127);
+    a.n_slots = (int)((budget - fixed) / slot_bytes);
+    if (a.n_slots > 8) a.n_slots = 8;
+    if (a.n_slots < 4) return SV_EUNSUPPORTED;
+    const size_t smem = fixed + (size_t)a.n_slots * slot_bytes;
+    if (cudaFuncSetAttribute(attn_tc_kernel<NQ, TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)smem) != cudaSuccess)
+        return SV_ECUDA;
+    attn_tc_kernel<NQ, TILE><<<grid, 128 + 128 * NQ, smem, stream>>>(a, p.pool->k_map, p.pool->v_map);
+    return launch_check();
 }
 
 sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t workspace_bytes,
@@ -795,28 +828,12 @@ sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t worksp
     a.n_pool_pages = p.pool->n_pages;
     a.group = p.hq / p.hkv;
     a.nq = rows_groups(p);
-    const int grid = sm_count();
+    const int grid = attn_grid(a.nq);
     if (workspace_bytes < prefix_bytes(p.batch) + (size_t)grid * 2 * part_slot_floats(a.nq) * sizeof(float))
         return SV_EWORKSPACE;
     a.ws_prefix = static_cast<int32_t *>(workspace);
     a.ws_part = reinterpret_cast<float *>(static_cast<uint8_t *>(workspace) + prefix_bytes(p.batch));
-    const size_t fixed = (size_t)a.nq * QGROUP_BYTES + sizeof(Shared) + 1024;
-    const size_t budget = 227 * 1024;
-    a.n_slots = (int)((budget - fixed) / SLOT_BYTES);
-    if (a.n_slots > 8) a.n_slots = 8;
-    if (a.n_slots < 4) return SV_EUNSUPPORTED;
-    const size_t smem = fixed + (size_t)a.n_slots * SLOT_BYTES;
-    cudaError_t e;
-    if (a.nq == 1) {
-        e = cudaFuncSetAttribute(attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return SV_ECUDA;
-        attn_tc_kernel<1><<<grid, 256, smem, stream>>>(a, p.pool->k_map, p.pool->v_map);
-    } else {
-        e = cudaFuncSetAttribute(attn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return SV_ECUDA;
-        attn_tc_kernel<2><<<grid, 384, smem, stream>>>(a, p.pool->k_map, p.pool->v_map);
-    }
-    sv_status st = launch_check();
+    sv_status st = a.nq == 1 ? launch_main<1, 64>(a, p, grid, stream) : launch_main<2, 128>(a, p, grid, stream);
     if (st != SV_OK) return st;
     attn_combine_kernel<<<p.batch * p.hkv, 256, 0, stream>>>(a);
     return launch_check();
