@@ -201,7 +201,7 @@ struct Shared {
     uint64_t empty[8];       // ring slot released by the tensor core
     uint64_t s_full[2];      // S accumulator ready
     uint64_t p_full[2];      // P written by the softmax threads
-    uint64_t o_done[2];      // PV of a row group finished
+    uint64_t o_done[2];      // PV of unit u finished (indexed by u & 1, like s_full / p_full)
     uint64_t q_full;         // query rows of a segment are in shared memory
     uint32_t tmem_base;
     int abort_flag;
@@ -476,7 +476,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                         for (int ks = 0; ks < TILE / 16; ++ks)
                             tc_mma_ts(d, pa + ks * 8, smem_desc(va + ks * 2048, SLOT_BYTES / 2, 1024),
                                       idesc_pv, (ti > 0 || ks > 0) ? 1u : 0u);
-                        tc_commit(smem_u32(&sh->o_done[q]));
+                        tc_commit(smem_u32(&sh->o_done[gu & 1]));
                         if (q == nq_seg - 1) tc_commit(smem_u32(&sh->empty[slot]));   // V tile consumed
                         if (u + 2 < n_units) issue_qk(u + 2);
                     }
@@ -500,7 +500,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
             const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
             TileCursor cur;
             cur.seek(p, sh, t_begin, TILE);
-            uint32_t ug = 0, kq = 0;       // global unit counter, units of this group so far
+            uint32_t ug = 0;               // global unit counter
             uint32_t seg_no = 0;
             bool ok = true;
             for (long long tg = t_begin; tg < t_end && ok; ++seg_no) {
@@ -554,7 +554,6 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     if (!ok) break;
                     if (!warp_active) {                         // all 32 rows are padding
                         mbar_arrive(smem_u32(&sh->p_full[gu & 1]));
-                        ++kq;
                         continue;
                     }
                     tc_fence_after();
@@ -589,14 +588,19 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                         }
                     }
                     const float m_use = (m_ref == -CUDART_INF_F) ? 0.f : m_ref;
-                    // previous PV of this row group must be complete before O may be touched;
-                    // waiting every time keeps the barrier's phase in step with kq
-                    if (kq > 0) ok = bounded_wait(smem_u32(&sh->o_done[q]), (kq - 1) & 1, sh, p.device_status);
-                    if (!ok) break;
                     if (rescale) l_sum *= factor;
                     // tensor-memory accesses are warp-wide: if any row of the warp has to rescale
                     // its accumulator, the whole warp goes through (factor 1 elsewhere)
                     if (__any_sync(0xffffffffu, rescale && ti > 0)) {
+                        // The accumulator may only be touched once the previous PV of this row
+                        // group is complete.  The tensor core runs in issue order (PV(u), then
+                        // QK(u+2)), so having seen S(gu) means PV(gu-2) is done: with two row
+                        // groups that IS the previous PV of this group; with one group it is
+                        // PV(gu-1), whose barrier is then at most one phase behind.
+                        if (nq_seg == 1)
+                            ok = bounded_wait(smem_u32(&sh->o_done[(gu - 1) & 1]), ((gu - 1) >> 1) & 1, sh,
+                                              p.device_status);
+                        if (!ok) break;
                         tc_fence_after();
                         const float f = (rescale && ti > 0) ? factor : 1.f;
 #pragma unroll
@@ -638,11 +642,14 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     tc_wait_st();
                     tc_fence_before();
                     mbar_arrive(smem_u32(&sh->p_full[gu & 1]));
-                    ++kq;
                 }
                 if (!ok) break;
                 // ---- epilogue of the segment: wait for the last PV, then read O
-                ok = bounded_wait(smem_u32(&sh->o_done[q]), (kq - 1) & 1, sh, p.device_status);
+                {
+                    const uint32_t gl = ug + (seg_tiles - 1) * nq_seg + q;     // this group's last unit
+                    if (warp_active)
+                        ok = bounded_wait(smem_u32(&sh->o_done[gl & 1]), (gl >> 1) & 1, sh, p.device_status);
+                }
                 if (!ok) break;
                 tc_fence_after();
                 const bool whole = (cur.t == 0 && seg_tiles == cur.n_tiles);
