@@ -75,6 +75,14 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map
         "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
         : "memory");
 }
+// true in exactly one lane of a converged warp; unlike `lane == 0` it keeps the surrounding
+// code warp-uniform for the compiler, so descriptors stay in uniform registers
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile("{\n .reg .pred P;\n elect.sync _|P, 0xffffffff;\n selp.u32 %0, 1, 0, P;\n}\n" : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar)
@@ -418,8 +426,11 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
             }
         } else if (t_end > t_begin && warp == 1) {
             // ================================================================ MMA issuer
-            if (lane == 0) {
+            // the whole warp walks the schedule and waits; one elected lane issues
+            {
                 const uint32_t idesc_qk = instr_desc(false, TILE), idesc_pv = instr_desc(true, HD);
+                const uint64_t q_desc0 = smem_desc(smem_u32(q_smem), 16, 1024);
+                const uint64_t q_desc1 = smem_desc(smem_u32(q_smem + (NQ - 1) * QGROUP_BYTES), 16, 1024);
                 TileCursor cur;
                 cur.seek(p, sh, t_begin, TILE);
                 uint32_t tile_no = 0;      // tiles of this block so far (ring position)
@@ -443,18 +454,21 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                             tc_fence_after();
                         }
                         if (!ok) return;
-                        const uint32_t ka = smem_u32(ring + slot * SLOT_BYTES);
-                        const uint32_t qa = smem_u32(q_smem + q * QGROUP_BYTES);
+                        // descriptors are built once; stepping along K only adds to the address field
+                        const uint64_t kd = smem_desc(smem_u32(ring + slot * SLOT_BYTES), 16, 1024);
+                        const uint64_t qd = q == 0 ? q_desc0 : q_desc1;
                         const uint32_t d = tmem + ((ug + u) & 1) * TILE;
+                        if (elect_one()) {
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {
-                            const uint32_t koff = (ks >> 2) * (SLOT_BYTES / 2) + (ks & 3) * 32;
-                            const uint32_t qoff = (ks >> 2) * (QGROUP_BYTES / 2) + (ks & 3) * 32;
-                            tc_mma_ss(d, smem_desc(qa + qoff, 16, 1024), smem_desc(ka + koff, 16, 1024),
-                                      idesc_qk, ks > 0);
+                            const uint32_t koff = ((ks >> 2) * (SLOT_BYTES / 2) + (ks & 3) * 32) >> 4;
+                            const uint32_t qoff = ((ks >> 2) * (QGROUP_BYTES / 2) + (ks & 3) * 32) >> 4;
+                            tc_mma_ss(d, qd + qoff, kd + koff, idesc_qk, ks > 0);
                         }
                         tc_commit(smem_u32(&sh->s_full[(ug + u) & 1]));
                         if (q == nq_seg - 1) tc_commit(smem_u32(&sh->empty[slot]));   // K tile consumed
+                        }
+                        __syncwarp();
                     };
                     issue_qk(0);
                     if (n_units > 1) issue_qk(1);
@@ -469,15 +483,18 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                                               p.device_status);
                         if (!ok) break;
                         tc_fence_after();
-                        const uint32_t va = smem_u32(ring + slot * SLOT_BYTES);
+                        const uint64_t vd = smem_desc(smem_u32(ring + slot * SLOT_BYTES), SLOT_BYTES / 2, 1024);
                         const uint32_t pa = tmem + (gu & 1) * TILE;      // P overlays S, TILE/2 columns
                         const uint32_t d = tmem + O_COL0 + q * 128;
+                        if (elect_one()) {
 #pragma unroll
                         for (int ks = 0; ks < TILE / 16; ++ks)
-                            tc_mma_ts(d, pa + ks * 8, smem_desc(va + ks * 2048, SLOT_BYTES / 2, 1024),
-                                      idesc_pv, (ti > 0 || ks > 0) ? 1u : 0u);
+                            tc_mma_ts(d, pa + ks * 8, vd + (uint64_t)(ks * (2048 >> 4)), idesc_pv,
+                                      (ti > 0 || ks > 0) ? 1u : 0u);
                         tc_commit(smem_u32(&sh->o_done[gu & 1]));
                         if (q == nq_seg - 1) tc_commit(smem_u32(&sh->empty[slot]));   // V tile consumed
+                        }
+                        __syncwarp();
                         if (u + 2 < n_units) issue_qk(u + 2);
                     }
                     ug += n_units;
