@@ -650,8 +650,17 @@ static sv_status launch_accept(const sv_accept_params *p, void *scratch, int sli
     a.n_seg = (p->vocab + SEG - 1) / SEG;
     a.vec_ok = (p->row_stride % 4 == 0) && aligned16(p->target_logits) &&
                (p->draft_logits == nullptr || aligned16(p->draft_logits));
-    // blocks per sequence in the float64 pass: enough to occupy the machine, at least 8 segments each
-    int splits = (4 * sm_count() + p->batch - 1) / p->batch;
+    // blocks per sequence in the float64 pass: fill the machine once (a second, nearly empty
+    // wave would double the time), at least 8 segments per block
+    static int seg_blocks_per_sm = 0;
+    if (seg_blocks_per_sm == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, accept_segsum_kernel, SEG_THREADS, 0) !=
+                cudaSuccess || n < 1)
+            n = 2;
+        seg_blocks_per_sm = n;
+    }
+    int splits = (seg_blocks_per_sm * sm_count()) / p->batch;
     if (splits > MAX_SPLITS) splits = MAX_SPLITS;
     if (splits > (a.n_seg + 7) / 8) splits = (a.n_seg + 7) / 8;
     if (splits < 1) splits = 1;

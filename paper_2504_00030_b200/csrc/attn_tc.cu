@@ -734,7 +734,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
 
 // ---------------------------------------------------------------------------- combine kernel
 // One block per (sequence, kv head); merges the partials of pairs whose tiles were shared
-// by several blocks of the main kernel.  Thread = query row.
+// by several blocks of the main kernel.  Warp = query row.
 __global__ void __launch_bounds__(256)
 attn_combine_kernel(const AttnTcLaunch a)
 {
@@ -755,42 +755,40 @@ attn_combine_kernel(const AttnTcLaunch a)
     int gam = p.gamma[b];
     gam = min(max(gam, 0), p.gamma_max);
     const int G = a.group, n_rows = G * (gam + 1);
-    for (int r = threadIdx.x; r < n_rows; r += blockDim.x) {
+    // one warp per query row: the lanes cover head_dim as float4, so every access is a full line
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const size_t m_off = (size_t)NQ * 128 * HD, l_off = m_off + (size_t)NQ * 128;
+    for (int r = warp; r < n_rows; r += n_warps) {
         float m = -CUDART_INF_F;
         for (long long c = c_first; c <= c_last; ++c) {
             if (share_begin(c + 1, total, grid) == share_begin(c, total, grid)) continue;   // empty share
             const int which = (share_begin(c, total, grid) >= T0) ? 0 : 1;
             const float *slot = a.ws_part + ((size_t)c * 2 + which) * part_slot_floats(NQ);
-            m = fmaxf(m, slot[(size_t)NQ * 128 * HD + r]);
+            m = fmaxf(m, slot[m_off + r]);
         }
-        float acc[HD];
-#pragma unroll
-        for (int d = 0; d < HD; ++d) acc[d] = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         float l = 0.f;
         for (long long c = c_first; c <= c_last; ++c) {
             if (share_begin(c + 1, total, grid) == share_begin(c, total, grid)) continue;
             const int which = (share_begin(c, total, grid) >= T0) ? 0 : 1;
             const float *slot = a.ws_part + ((size_t)c * 2 + which) * part_slot_floats(NQ);
-            const float mc = slot[(size_t)NQ * 128 * HD + r];
+            const float mc = slot[m_off + r];
             if (mc == -CUDART_INF_F) continue;
             const float w = exp2f(mc - m);
-            l += w * slot[(size_t)NQ * 128 * HD + NQ * 128 + r];
-            const float4 *orow = reinterpret_cast<const float4 *>(slot + (size_t)r * HD);
-#pragma unroll
-            for (int d = 0; d < HD / 4; ++d) {
-                const float4 v = orow[d];
-                acc[4 * d] += w * v.x; acc[4 * d + 1] += w * v.y;
-                acc[4 * d + 2] += w * v.z; acc[4 * d + 3] += w * v.w;
-            }
+            l += w * slot[l_off + r];
+            const float4 v = reinterpret_cast<const float4 *>(slot + (size_t)r * HD)[lane];
+            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
         }
         const int i = r / G, hh = r - i * G;
         const long long q_row = ((long long)p.cu_q[b] + i) * p.hq + (long long)g * G + hh;
         const float inv = 1.f / l;
-        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.o) + q_row * HD;
-#pragma unroll
-        for (int d = 0; d < HD; d += 2)
-            *reinterpret_cast<__nv_bfloat162 *>(dst + d) = __floats2bfloat162_rn(acc[d] * inv, acc[d + 1] * inv);
-        if (p.lse != nullptr) p.lse[q_row] = (m + log2f(l)) * 0.6931471805599453f;
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+        uint2 packed;
+        packed.x = *reinterpret_cast<const uint32_t *>(&lo);
+        packed.y = *reinterpret_cast<const uint32_t *>(&hi);
+        reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.o) + q_row * HD)[lane] = packed;
+        if (lane == 0 && p.lse != nullptr) p.lse[q_row] = (m + log2f(l)) * 0.6931471805599453f;
     }
 }
 
