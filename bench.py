@@ -30,7 +30,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2504_00030_b200 import synth  # noqa: E402
+from paper_2504_00030_b200 import shard, synth  # noqa: E402
 
 METRIC = "verified tokens/sec (verify step: attention + accept/resample + gamma update)"
 UNIT = "tokens/s"
@@ -46,7 +46,7 @@ def measured_peaks():
 
 
 def workload_inputs(cfg, rank, batch=None, gamma=None, gamma_max=None):
-    cfg = synth.scaled(cfg, seed=cfg.seed + 1000 * rank)
+    cfg = synth.scaled(cfg, seed=shard.rank_seed(cfg.seed, rank))
     if gamma_max is not None:
         cfg = synth.scaled(cfg, gamma_max=gamma_max)
     if gamma is not None:
@@ -326,15 +326,7 @@ def run_ours(args):
     assert e2e_tokens == tokens
 
     # ---- reduce over ranks: max time, sum of tokens
-    if world > 1:
-        t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=DEV)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, e2e_ms = float(t[0]), float(t[1])
-        c = torch.tensor([tokens], dtype=torch.int64, device=DEV)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        tokens_all = int(c[0])
-    else:
-        tokens_all = tokens
+    (ms_total, e2e_ms), tokens_all = shard.reduce_timing([ms_total, e2e_ms], tokens, device=DEV)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
