@@ -22,187 +22,21 @@
 // Warps: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 4..7 = softmax / epilogue of row
 // group 0, 8..11 = row group 1 (when needed).  All hand-offs are mbarriers; every wait is
 // bounded and an expired wait sets SV_DEV_TIMEOUT and drains the block.
-#include "attn_common.cuh"
+#include "attn_sched.cuh"
+#include "tc_ptx.cuh"
 
 #include <math_constants.h>
+#include <stdlib.h>
 
 namespace sv {
 
-constexpr int HD = 128;                 // head_dim of this kernel
 // Tokens per key tile are a template parameter: 64 (4 pages, 16 KB per K or V tile) when one
 // row group suffices -- two thread blocks then share an SM and hide each other's hand-off
 // latencies -- and 128 (8 pages, 32 KB) with two row groups, one block per SM.
 constexpr int QGROUP_BYTES = 128 * HD * 2;         // 32 KB: 128 query rows
-constexpr int MAX_BATCH_TC = 1 << 20;
-constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2 s: far beyond any legitimate wait
 constexpr float RESCALE_THRESHOLD = 8.f;           // log2 units: P <= 2^8 before a lazy rescale
 
-// ---------------------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p)
-{
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        " selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, int c0, int c1,
-                                            int c2, int c3, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
-        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
-        : "memory");
-}
-// true in exactly one lane of a converged warp; unlike `lane == 0` it keeps the surrounding
-// code warp-uniform for the compiler, so descriptors stay in uniform registers
-__device__ __forceinline__ bool elect_one()
-{
-    uint32_t pred;
-    asm volatile("{\n .reg .pred P;\n elect.sync _|P, 0xffffffff;\n selp.u32 %0, 1, 0, P;\n}\n" : "=r"(pred));
-    return pred != 0;
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-                 : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate)
-{
-    asm volatile(
-        "{\n .reg .pred p;\n setp.ne.u32 p, %4, 0;\n"
-        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate)
-{
-    asm volatile(
-        "{\n .reg .pred p;\n setp.ne.u32 p, %4, 0;\n"
-        " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(d),
-        "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// 32 consecutive fp32 columns of this thread's TMEM lane
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
-          "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
-          "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
-          "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-// same without the wait: several loads can be in flight, then one tc_wait_ld()
-__device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t *r)
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
-          "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
-          "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
-          "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
-        "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
-        "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-        : "memory");
-}
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// Shared-memory matrix descriptor, 128-byte swizzle.  Tiles are stored as two 16 KB halves
-// (64 of the 128 dims each), each half as rows of 128 bytes (one token or one query row),
-// groups of 8 rows = 1024 bytes.
-//   K-major (Q as A, K as B): stride between 8-row groups = 1024; leading offset unused.
-//   N-major (V as B, N = dim): the 8 K-rows (tokens) of a group are 128 bytes apart, groups
-//   1024 bytes apart (stride offset), the second 64 dims 16 KB further (leading offset).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-    d |= (uint64_t)1 << 46;      // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;      // 128-byte swizzle
-    return d;
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n.
-__device__ __forceinline__ uint32_t instr_desc(bool b_n_major, int n)
-{
-    uint32_t d = 0;
-    d |= 1u << 4;                 // accumulator fp32
-    d |= 1u << 7;                 // A bf16
-    d |= 1u << 10;                // B bf16
-    d |= (b_n_major ? 1u : 0u) << 16;
-    d |= (uint32_t)(n >> 3) << 17;
-    d |= (uint32_t)(128 >> 4) << 24;
-    return d;
-}
-
-// ---------------------------------------------------------------------------- schedule
-struct AttnTcLaunch {
-    sv_attn_params p;
-    int64_t n_pool_pages;
-    int group;           // query heads per kv head
-    int nq;              // row groups of 128 rows (1 or 2)
-    int n_slots;         // K/V ring slots
-    int32_t *ws_prefix;  // [batch+1] tile prefix, then [2]: total tiles, grid size
-    float *ws_part;      // partial results: slot-major
-};
-
-__host__ __device__ inline size_t part_slot_floats(int nq) { return (size_t)nq * 128 * (HD + 2); }
-
-// first global tile of block c when `total` tiles are split over `grid` blocks
-__device__ __forceinline__ long long share_begin(long long c, long long total, long long grid)
-{
-    return (c * total) / grid;
-}
 
 struct Shared {
     uint64_t full[8];        // ring slot filled by TMA
@@ -218,64 +52,7 @@ struct Shared {
     int start_prefix;        // tiles (per kv head) of the sequences before it
 };
 
-__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, Shared *sh, uint32_t *status)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-#pragma unroll 1
-        for (int it = 0; it < 256; ++it)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*(volatile int *)&sh->abort_flag) return false;
-        if (clock64() - t0 > WAIT_CYCLES) break;
-    }
-    *(volatile int *)&sh->abort_flag = 1;
-    set_status(status, SV_DEV_TIMEOUT);
-    return false;
-}
 
-// Tiles and validated gamma of one sequence; sequences with inconsistent lengths own no tiles.
-__device__ __forceinline__ int seq_tiles(const sv_attn_params &p, int b, int *gam_out, bool report, int tile)
-{
-    int g = p.gamma[b];
-    if (g < 0 || g > p.gamma_max) {
-        if (report) set_status(p.device_status, SV_DEV_BAD_GAMMA);
-        g = min(max(g, 0), p.gamma_max);
-    }
-    const int L = p.seq_len[b];
-    int nt = (L + tile - 1) / tile;
-    if (L < g + 1 || (long long)(L + 15) / 16 > p.block_table_stride || L > p.max_seq_len) {
-        if (report) set_status(p.device_status, SV_DEV_BAD_LEN);
-        nt = 0;
-    }
-    if (gam_out != nullptr) *gam_out = g;
-    return nt;
-}
-
-// Walks the (sequence, kv head, tile) triples of a block's share.
-struct TileCursor {
-    int b, g, t, n_tiles, gam;    // current pair, tile inside it, its tile count and gamma
-    int tile_tokens;
-    __device__ void seek(const sv_attn_params &p, const Shared *sh, long long tile, int tokens)
-    {
-        tile_tokens = tokens;
-        b = sh->start_b;
-        n_tiles = seq_tiles(p, b, &gam, false, tile_tokens);
-        const long long rel = tile - (long long)sh->start_prefix * p.hkv;
-        g = (int)(rel / n_tiles);
-        t = (int)(rel % n_tiles);
-    }
-    __device__ void next_pair(const sv_attn_params &p)
-    {
-        t = 0;
-        if (++g == p.hkv) {
-            g = 0;
-            n_tiles = 0;
-            while (n_tiles == 0 && ++b < p.batch) n_tiles = seq_tiles(p, b, &gam, false, tile_tokens);
-            if (b >= p.batch) n_tiles = 1;      // past the end: never used
-        }
-    }
-};
 
 // ---------------------------------------------------------------------------- main kernel
 template <int NQ, int TILE>
@@ -387,7 +164,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
         if (t_end > t_begin && warp == 0) {
             // ================================================================ TMA producer
             TileCursor cur;
-            cur.seek(p, sh, t_begin, TILE);
+            cur.seek(p, sh->start_b, sh->start_prefix, t_begin, TILE);
             uint32_t item = 0;     // ring items: 2*tile = K, 2*tile+1 = V
             for (long long tg = t_begin; tg < t_end; ++tg) {
                 const int b = cur.b;
@@ -409,7 +186,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     const uint32_t slot = item % (uint32_t)n_slots;
                     const uint32_t use = item / (uint32_t)n_slots;
                     const uint32_t full = smem_u32(&sh->full[slot]);
-                    if (use > 0) ok = ok && bounded_wait(smem_u32(&sh->empty[slot]), (use - 1) & 1, sh, p.device_status);
+                    if (use > 0) ok = ok && bounded_wait(smem_u32(&sh->empty[slot]), (use - 1) & 1, &sh->abort_flag, p.device_status);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     if (lane == 0) mbar_expect_tx(full, SLOT_BYTES);
@@ -432,7 +209,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 const uint64_t q_desc0 = smem_desc(smem_u32(q_smem), 16, 1024);
                 const uint64_t q_desc1 = smem_desc(smem_u32(q_smem + (NQ - 1) * QGROUP_BYTES), 16, 1024);
                 TileCursor cur;
-                cur.seek(p, sh, t_begin, TILE);
+                cur.seek(p, sh->start_b, sh->start_prefix, t_begin, TILE);
                 uint32_t tile_no = 0;      // tiles of this block so far (ring position)
                 uint32_t ug = 0;           // global unit counter: unit = (tile, row group)
                 uint32_t seg_no = 0;
@@ -442,14 +219,14 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     // row groups this pair really has (a second group only if it has > 128 rows)
                     const int nq_seg = (NQ == 2 && G * (cur.gam + 1) > 128) ? 2 : 1;
                     const int n_units = seg_tiles * nq_seg;
-                    ok = bounded_wait(smem_u32(&sh->q_full), seg_no & 1, sh, p.device_status);
+                    ok = bounded_wait(smem_u32(&sh->q_full), seg_no & 1, &sh->abort_flag, p.device_status);
                     tc_fence_after();
                     auto issue_qk = [&](int u) {       // unit u of this segment
                         const int q = u % nq_seg, ti = u / nq_seg;
                         const uint32_t item = 2 * (tile_no + ti);
                         const uint32_t slot = item % (uint32_t)n_slots;
                         if (q == 0) {
-                            ok = ok && bounded_wait(smem_u32(&sh->full[slot]), (item / n_slots) & 1, sh,
+                            ok = ok && bounded_wait(smem_u32(&sh->full[slot]), (item / n_slots) & 1, &sh->abort_flag,
                                                     p.device_status);
                             tc_fence_after();
                         }
@@ -475,11 +252,11 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     for (int u = 0; u < n_units && ok; ++u) {
                         const int q = u % nq_seg, ti = u / nq_seg;
                         const uint32_t gu = ug + u;
-                        ok = bounded_wait(smem_u32(&sh->p_full[gu & 1]), (gu >> 1) & 1, sh, p.device_status);
+                        ok = bounded_wait(smem_u32(&sh->p_full[gu & 1]), (gu >> 1) & 1, &sh->abort_flag, p.device_status);
                         const uint32_t item = 2 * (tile_no + ti) + 1;
                         const uint32_t slot = item % (uint32_t)n_slots;
                         if (ok && q == 0)
-                            ok = bounded_wait(smem_u32(&sh->full[slot]), (item / n_slots) & 1, sh,
+                            ok = bounded_wait(smem_u32(&sh->full[slot]), (item / n_slots) & 1, &sh->abort_flag,
                                               p.device_status);
                         if (!ok) break;
                         tc_fence_after();
@@ -516,7 +293,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
             const int r = q * 128 + r_in;                      // row of the (b, g) pair
             const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
             TileCursor cur;
-            cur.seek(p, sh, t_begin, TILE);
+            cur.seek(p, sh->start_b, sh->start_prefix, t_begin, TILE);
             uint32_t ug = 0;               // global unit counter
             uint32_t seg_no = 0;
             bool ok = true;
@@ -551,10 +328,10 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     // Stay in step with the barriers this group will use again later: a parity
                     // wait is only meaningful for a waiter that is at most one phase ahead, so the
                     // idle group follows every phase of q_full and of both s_full barriers.
-                    ok = bounded_wait(smem_u32(&sh->q_full), seg_no & 1, sh, p.device_status);
+                    ok = bounded_wait(smem_u32(&sh->q_full), seg_no & 1, &sh->abort_flag, p.device_status);
                     for (int ti = 0; ti < seg_tiles && ok; ++ti) {
                         const uint32_t gu = ug + ti;            // nq_seg == 1 here
-                        ok = bounded_wait(smem_u32(&sh->s_full[gu & 1]), (gu >> 1) & 1, sh, p.device_status);
+                        ok = bounded_wait(smem_u32(&sh->s_full[gu & 1]), (gu >> 1) & 1, &sh->abort_flag, p.device_status);
                     }
                     ug += seg_tiles * nq_seg;
                     tg += seg_tiles;
@@ -567,7 +344,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 for (int ti = 0; ti < seg_tiles && ok; ++ti) {
                     const uint32_t gu = ug + ti * nq_seg + q;
                     const uint32_t s_addr = tmem + lane_addr + (gu & 1) * TILE;
-                    ok = bounded_wait(smem_u32(&sh->s_full[gu & 1]), (gu >> 1) & 1, sh, p.device_status);
+                    ok = bounded_wait(smem_u32(&sh->s_full[gu & 1]), (gu >> 1) & 1, &sh->abort_flag, p.device_status);
                     if (!ok) break;
                     if (!warp_active) {                         // all 32 rows are padding
                         mbar_arrive(smem_u32(&sh->p_full[gu & 1]));
@@ -615,7 +392,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                         // groups that IS the previous PV of this group; with one group it is
                         // PV(gu-1), whose barrier is then at most one phase behind.
                         if (nq_seg == 1)
-                            ok = bounded_wait(smem_u32(&sh->o_done[(gu - 1) & 1]), ((gu - 1) >> 1) & 1, sh,
+                            ok = bounded_wait(smem_u32(&sh->o_done[(gu - 1) & 1]), ((gu - 1) >> 1) & 1, &sh->abort_flag,
                                               p.device_status);
                         if (!ok) break;
                         tc_fence_after();
@@ -665,7 +442,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 {
                     const uint32_t gl = ug + (seg_tiles - 1) * nq_seg + q;     // this group's last unit
                     if (warp_active)
-                        ok = bounded_wait(smem_u32(&sh->o_done[gl & 1]), (gl >> 1) & 1, sh, p.device_status);
+                        ok = bounded_wait(smem_u32(&sh->o_done[gl & 1]), (gl >> 1) & 1, &sh->abort_flag, p.device_status);
                 }
                 if (!ok) break;
                 tc_fence_after();
@@ -698,7 +475,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                         p.lse[q_row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
                 } else {
                     // partial: fp32 O row, then max and sum; slot 0 = the block's first segment
-                    float *slot = a.ws_part + ((size_t)blockIdx.x * 2 + (seg_no == 0 ? 0 : 1)) * part_slot_floats(NQ);
+                    float *slot = a.ws_part + ((size_t)blockIdx.x * 2 + (seg_no == 0 ? 0 : 1)) * part_slot_floats(NQ * 128);
                     float *orow = slot + (size_t)r * HD;
 #pragma unroll
                     for (int ch = 0; ch < 4; ++ch) {
@@ -740,7 +517,7 @@ attn_combine_kernel(const AttnTcLaunch a)
 {
     const sv_attn_params &p = a.p;
     const int b = blockIdx.x / p.hkv, g = blockIdx.x % p.hkv;
-    const int NQ = a.nq;
+    const int slot_rows = a.slot_rows;
     const long long grid = a.ws_prefix[p.batch + 1];
     const long long total = (long long)a.ws_prefix[p.batch] * p.hkv;
     const int n_tiles = a.ws_prefix[b + 1] - a.ws_prefix[b];
@@ -757,13 +534,13 @@ attn_combine_kernel(const AttnTcLaunch a)
     const int G = a.group, n_rows = G * (gam + 1);
     // one warp per query row: the lanes cover head_dim as float4, so every access is a full line
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    const size_t m_off = (size_t)NQ * 128 * HD, l_off = m_off + (size_t)NQ * 128;
+    const size_t m_off = (size_t)slot_rows * HD, l_off = m_off + (size_t)slot_rows;
     for (int r = warp; r < n_rows; r += n_warps) {
         float m = -CUDART_INF_F;
         for (long long c = c_first; c <= c_last; ++c) {
             if (share_begin(c + 1, total, grid) == share_begin(c, total, grid)) continue;   // empty share
             const int which = (share_begin(c, total, grid) >= T0) ? 0 : 1;
-            const float *slot = a.ws_part + ((size_t)c * 2 + which) * part_slot_floats(NQ);
+            const float *slot = a.ws_part + ((size_t)c * 2 + which) * part_slot_floats(slot_rows);
             m = fmaxf(m, slot[m_off + r]);
         }
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -771,7 +548,7 @@ attn_combine_kernel(const AttnTcLaunch a)
         for (long long c = c_first; c <= c_last; ++c) {
             if (share_begin(c + 1, total, grid) == share_begin(c, total, grid)) continue;
             const int which = (share_begin(c, total, grid) >= T0) ? 0 : 1;
-            const float *slot = a.ws_part + ((size_t)c * 2 + which) * part_slot_floats(NQ);
+            const float *slot = a.ws_part + ((size_t)c * 2 + which) * part_slot_floats(slot_rows);
             const float mc = slot[m_off + r];
             if (mc == -CUDART_INF_F) continue;
             const float w = exp2f(mc - m);
@@ -820,7 +597,7 @@ size_t attn_tc_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t hq, int
     const int rows = (hq / hkv) * (gamma_max + 1);
     const int nq = (rows + 127) / 128;
     if (nq < 1 || nq > 2 || batch > MAX_BATCH_TC) return 0;
-    return prefix_bytes(batch) + (size_t)attn_grid(nq) * 2 * part_slot_floats(nq) * sizeof(float);
+    return prefix_bytes(batch) + (size_t)attn_grid(nq) * 2 * part_slot_floats(nq * 128) * sizeof(float);
 }
 
 template <int NQ, int TILE>
@@ -842,6 +619,18 @@ static sv_status launch_main(AttnTcLaunch &a, const sv_attn_params &p, int grid,
     return launch_check();
 }
 
+// 0 = pick by shape, 1 = always the shared-memory-Q kernels of this file, 2 = the
+// tensor-memory-Q kernel whenever it supports the shape.  Read once from SV_ATTN_VARIANT
+// (a diagnostic switch; both choices compute the same thing).
+static int attn_variant()
+{
+    static const int v = [] {
+        const char *e = getenv("SV_ATTN_VARIANT");
+        return (e != nullptr && e[0] >= '0' && e[0] <= '2') ? e[0] - '0' : 0;
+    }();
+    return v;
+}
+
 sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t workspace_bytes,
                          cudaStream_t stream)
 {
@@ -850,12 +639,18 @@ sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t worksp
     a.n_pool_pages = p.pool->n_pages;
     a.group = p.hq / p.hkv;
     a.nq = rows_groups(p);
-    const int grid = attn_grid(a.nq);
-    if (workspace_bytes < prefix_bytes(p.batch) + (size_t)grid * 2 * part_slot_floats(a.nq) * sizeof(float))
+    const int rows = a.group * (p.gamma_max + 1);
+    const int variant = attn_variant();
+    const bool use_tq = attn_tq_supported(p) && variant != 1;
+    a.slot_rows = use_tq ? attn_tq_slot_rows(rows) : a.nq * 128;
+    const int grid = use_tq ? sm_count() : attn_grid(a.nq);
+    if (workspace_bytes < prefix_bytes(p.batch) + (size_t)grid * 2 * part_slot_floats(a.slot_rows) * sizeof(float))
         return SV_EWORKSPACE;
     a.ws_prefix = static_cast<int32_t *>(workspace);
     a.ws_part = reinterpret_cast<float *>(static_cast<uint8_t *>(workspace) + prefix_bytes(p.batch));
-    sv_status st = a.nq == 1 ? launch_main<1, 64>(a, p, grid, stream) : launch_main<2, 128>(a, p, grid, stream);
+    sv_status st;
+    if (use_tq) st = launch_attn_tq_main(a, p, grid, stream);
+    else st = a.nq == 1 ? launch_main<1, 64>(a, p, grid, stream) : launch_main<2, 128>(a, p, grid, stream);
     if (st != SV_OK) return st;
     attn_combine_kernel<<<p.batch * p.hkv, 256, 0, stream>>>(a);
     return launch_check();

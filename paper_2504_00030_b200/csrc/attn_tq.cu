@@ -1,0 +1,785 @@
+// Draft-block attention, "queries in tensor memory" variant (tcgen05, sm_100a).
+//
+// Same schedule and data path as attn_tc.cu (stream-K over 128-token key tiles, TMA-staged
+// pages, S = Q K^T and O += P V on the tensor cores with accumulators in tensor memory), with
+// two changes that matter when a (sequence, kv head) pair has up to 144 query rows:
+//
+//  * The 128 query rows of the first row group live in TENSOR memory (64 columns of bf16
+//    pairs) and enter S = Q K^T as the A operand from there.  Shared memory then holds nothing
+//    but the K/V ring -- six or seven 32 KB slots, i.e. three or more tiles in flight per SM,
+//    which is what the HBM latency asks for -- and the Q K^T instructions cost about a third
+//    less than with A in shared memory.
+//  * Rows 128..143 (8 query heads x 17 positions = 136 rows is the case that matters) do not
+//    get a second 128-row tensor-memory group, whose instructions would cost as much as the
+//    first group's for 1/16 of the useful work.  Four extra warps take them with warp-level
+//    mma.sync (m16n8k16): each warp owns 32 of a tile's 128 tokens, reads the same K/V
+//    shared-memory tiles with ldmatrix, keeps its own running max / sum / fp32 O (16 x 128) in
+//    registers, and the four partial states are merged through shared memory when the
+//    segment ends.
+//
+// Warps: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 4..7 = softmax / epilogue of rows
+// 0..127 (thread = row = TMEM lane), 8..11 = tail rows (template parameter TAIL).  All
+// hand-offs are mbarriers; every wait is bounded, an expired wait sets SV_DEV_TIMEOUT and
+// drains the block.
+#include "attn_sched.cuh"
+#include "tc_ptx.cuh"
+
+#include <math_constants.h>
+
+namespace sv {
+
+namespace tq {
+
+constexpr int TILE = 128;                          // tokens per key tile
+constexpr int SLOT_BYTES = TILE * HD * 2;          // one K or one V tile: 32 KB
+constexpr int S_COL0 = 0;                          // TMEM columns: two S buffers,
+constexpr int O_COL0 = 256;                        // the O accumulator,
+constexpr int Q_COL0 = 384;                        // the query rows (bf16 pairs)
+constexpr uint32_t TMEM_COLS = 512;
+constexpr int TAIL_ROWS = 16;
+constexpr float RESCALE_THRESHOLD = 8.f;           // log2 units: P <= 2^8 before a lazy rescale
+
+struct Shared {
+    uint64_t full[8];        // ring slot filled by TMA
+    uint64_t empty[8];       // ring slot released by all its readers
+    uint64_t s_full[2];      // S accumulator ready
+    uint64_t p_full[2];      // P written by the softmax threads
+    uint64_t o_done[2];      // PV of tile u finished (indexed by u & 1)
+    uint64_t q_full;         // query rows of a segment are in tensor memory
+    uint64_t tail_sync;      // the four tail warps meet here around their merge
+    uint32_t tmem_base;
+    int abort_flag;
+    int total_tiles;
+    int start_b;
+    int start_prefix;
+};
+
+// merge buffers of the tail warps: [warp][row][dim], then running max and sum [warp][row]
+struct TailMerge {
+    float o[4][TAIL_ROWS][HD];
+    float m[4][TAIL_ROWS];
+    float l[4][TAIL_ROWS];
+};
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2,
+                                                  uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+// D (16x8 fp32) += A (16x16 bf16, row) * B (16x8 bf16, col)
+__device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+
+}  // namespace tq
+
+using namespace tq;
+
+template <bool TAIL>
+__global__ void __launch_bounds__(TAIL ? 384 : 256, 1)
+attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
+               const __grid_constant__ CUtensorMap v_map)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    // carve: [ring slots][tail merge buffers][Shared]; the swizzled tiles need a 1024-byte aligned base
+    uint8_t *ring = smem_raw;
+    if ((smem_u32(ring) & 1023u) != 0) {               // never seen; refuse rather than compute garbage
+        if (threadIdx.x == 0) set_status(a.p.device_status, SV_DEV_TIMEOUT);
+        return;
+    }
+    const int n_slots = a.n_slots;
+    TailMerge *tm = reinterpret_cast<TailMerge *>(ring + (size_t)n_slots * SLOT_BYTES);
+    Shared *sh = reinterpret_cast<Shared *>(ring + (size_t)n_slots * SLOT_BYTES + (TAIL ? sizeof(TailMerge) : 0));
+
+    const sv_attn_params &p = a.p;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int batch = p.batch, hkv = p.hkv, G = a.group;
+
+    if (tid == 0) {
+        for (int i = 0; i < n_slots; ++i) {
+            mbar_init(smem_u32(&sh->full[i]), 1);
+            mbar_init(smem_u32(&sh->empty[i]), TAIL ? 5 : 1);    // tensor core + one lane per tail warp
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&sh->s_full[i]), 1);
+            mbar_init(smem_u32(&sh->p_full[i]), 128);
+            mbar_init(smem_u32(&sh->o_done[i]), 1);
+        }
+        mbar_init(smem_u32(&sh->q_full), 128);
+        mbar_init(smem_u32(&sh->tail_sync), 4);
+        sh->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 0) {
+        // pass 1: total tiles; block 0 also publishes the inclusive prefix for the combine kernel
+        int carry = 0;
+        if (blockIdx.x == 0 && lane == 0) a.ws_prefix[0] = 0;
+        for (int base = 0; base < batch; base += 32) {
+            const int b = base + lane;
+            int v = (b < batch) ? seq_tiles(p, b, nullptr, blockIdx.x == 0, TILE) : 0;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, v, d);
+                if (lane >= d) v += t;
+            }
+            if (blockIdx.x == 0 && b < batch) a.ws_prefix[b + 1] = carry + v;
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+        const long long total = (long long)carry * hkv;
+        const long long my_begin = share_begin(blockIdx.x, total, gridDim.x);
+        if (lane == 0) {
+            sh->total_tiles = carry;
+            sh->start_b = 0;
+            sh->start_prefix = 0;
+            if (blockIdx.x == 0) a.ws_prefix[batch + 1] = (int)gridDim.x;
+        }
+        __syncwarp();
+        // pass 2: the sequence whose tiles contain this block's first tile
+        carry = 0;
+        for (int base = 0; base < batch; base += 32) {
+            const int b = base + lane;
+            const int nt = (b < batch) ? seq_tiles(p, b, nullptr, false, TILE) : 0;
+            int v = nt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, v, d);
+                if (lane >= d) v += t;
+            }
+            const long long lo = (long long)(carry + v - nt) * hkv, hi = (long long)(carry + v) * hkv;
+            if (nt > 0 && lo <= my_begin && my_begin < hi) {
+                sh->start_b = b;
+                sh->start_prefix = carry + v - nt;
+            }
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(&sh->tmem_base)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    const long long total = (long long)sh->total_tiles * hkv;
+    const long long grid = gridDim.x;
+    const long long t_begin = share_begin(blockIdx.x, total, grid);
+    const long long t_end = share_begin(blockIdx.x + 1, total, grid);
+    const uint32_t tmem = sh->tmem_base;
+    const float c_scale = p.sm_scale * 1.4426950408889634f;   // scores in log2 units
+    const int start_b = sh->start_b, start_prefix = sh->start_prefix;
+    int *abort_flag = &sh->abort_flag;
+
+    // With the tail warps there are 384 threads and 168 registers each at launch; the producer /
+    // MMA warpgroup hands most of its share to the others (128 * (80 + 208 + 216) = 384 * 168).
+    if (warp < 4) {
+        if (TAIL) asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+        if (t_end > t_begin && warp != 1) {
+            // ================================================================ TMA producers
+            // One thread gets a tensor copy under way every ~90 cycles, and a tile needs 32 of
+            // them (K and V, 8 pages, two 64-dim halves): one warp cannot keep up with HBM.  Warps
+            // 0, 2 and 3 therefore take the ring items (2*tile = K, 2*tile+1 = V) round robin.
+            const int pi = warp == 0 ? 0 : warp - 1;       // producer index 0..2
+            TileCursor cur;
+            cur.seek(p, start_b, start_prefix, t_begin, TILE);
+            const int page_in_tile = (lane >> 1) & 7, half = lane & 1;   // lane l < 16: page l/2, dims half l%2
+            bool ok = true;
+            long long tg = t_begin;
+            for (uint32_t item = pi; ok && t_begin + (item >> 1) < t_end; item += 3) {
+                while (tg < t_begin + (item >> 1)) {           // advance the cursor to this item's tile
+                    ++tg;
+                    if (++cur.t == cur.n_tiles) cur.next_pair(p);
+                }
+                const int b = cur.b;
+                const int L = p.seq_len[b];
+                const int n_pages = (L + 15) >> 4;
+                const int32_t *bt = p.block_table + (long long)b * p.block_table_stride;
+                const int lp = cur.t * (TILE / 16) + page_in_tile;
+                int phys = (int)a.n_pool_pages;       // out of range: TMA fills zeros, no traffic
+                if (lp < n_pages) {
+                    const int e = bt[lp];
+                    if (e < 0 || e >= a.n_pool_pages) set_status(p.device_status, SV_DEV_BAD_PAGE);
+                    else phys = e;
+                }
+                const uint32_t slot = item % (uint32_t)n_slots;
+                const uint32_t use = item / (uint32_t)n_slots;
+                const uint32_t full = smem_u32(&sh->full[slot]);
+                if (use > 0) ok = bounded_wait(smem_u32(&sh->empty[slot]), (use - 1) & 1, abort_flag, p.device_status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (lane == 0) mbar_expect_tx(full, SLOT_BYTES);
+                __syncwarp();
+                if (lane < 16) {
+                    const uint32_t dst = smem_u32(ring + slot * SLOT_BYTES + half * (SLOT_BYTES / 2) +
+                                                  page_in_tile * 2048);
+                    tma_load_4d(dst, (item & 1) == 0 ? &k_map : &v_map, half * 64, 0, cur.g, phys, full);
+                }
+            }
+        } else if (t_end > t_begin && warp == 1) {
+            // ================================================================ MMA issuer
+            // the whole warp walks the schedule and waits; one elected lane issues
+            const uint32_t idesc_qk = instr_desc(false, TILE), idesc_pv = instr_desc(true, HD);
+            TileCursor cur;
+            cur.seek(p, start_b, start_prefix, t_begin, TILE);
+            uint32_t tile_no = 0;      // tiles of this block so far (ring position and S / P buffer parity)
+            uint32_t seg_no = 0;
+            bool ok = true;
+            for (long long tg = t_begin; tg < t_end && ok;) {
+                const int seg_tiles = (int)min((long long)(cur.n_tiles - cur.t), t_end - tg);
+                ok = bounded_wait(smem_u32(&sh->q_full), seg_no & 1, abort_flag, p.device_status);
+                tc_fence_after();
+                auto issue_qk = [&](int ti) {
+                    const uint32_t gu = tile_no + ti;
+                    const uint32_t item = 2 * gu;
+                    const uint32_t slot = item % (uint32_t)n_slots;
+                    ok = ok && bounded_wait(smem_u32(&sh->full[slot]), (item / n_slots) & 1, abort_flag,
+                                            p.device_status);
+                    if (!ok) return;
+                    tc_fence_after();
+                    const uint64_t kd = smem_desc(smem_u32(ring + slot * SLOT_BYTES), 16, 1024);
+                    const uint32_t d = tmem + S_COL0 + (gu & 1) * TILE;
+                    if (elect_one()) {
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            const uint32_t koff = ((ks >> 2) * (SLOT_BYTES / 2) + (ks & 3) * 32) >> 4;
+                            tc_mma_ts(d, tmem + Q_COL0 + ks * 8, kd + koff, idesc_qk, ks > 0);
+                        }
+                        tc_commit(smem_u32(&sh->s_full[gu & 1]));
+                        tc_commit(smem_u32(&sh->empty[slot]));          // K tile consumed
+                    }
+                    __syncwarp();
+                };
+                issue_qk(0);
+                if (seg_tiles > 1) issue_qk(1);
+                for (int ti = 0; ti < seg_tiles && ok; ++ti) {
+                    const uint32_t gu = tile_no + ti;
+                    ok = bounded_wait(smem_u32(&sh->p_full[gu & 1]), (gu >> 1) & 1, abort_flag, p.device_status);
+                    const uint32_t item = 2 * gu + 1;
+                    const uint32_t slot = item % (uint32_t)n_slots;
+                    if (ok) ok = bounded_wait(smem_u32(&sh->full[slot]), (item / n_slots) & 1, abort_flag, p.device_status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t vd = smem_desc(smem_u32(ring + slot * SLOT_BYTES), SLOT_BYTES / 2, 1024);
+                    const uint32_t pa = tmem + S_COL0 + (gu & 1) * TILE;      // P overlays S, TILE/2 columns
+                    const uint32_t d = tmem + O_COL0;
+                    if (elect_one()) {
+#pragma unroll
+                        for (int ks = 0; ks < TILE / 16; ++ks)
+                            tc_mma_ts(d, pa + ks * 8, vd + (uint64_t)(ks * (2048 >> 4)), idesc_pv,
+                                      (ti > 0 || ks > 0) ? 1u : 0u);
+                        tc_commit(smem_u32(&sh->o_done[gu & 1]));
+                        tc_commit(smem_u32(&sh->empty[slot]));          // V tile consumed
+                    }
+                    __syncwarp();
+                    if (ti + 2 < seg_tiles) issue_qk(ti + 2);
+                }
+                tile_no += seg_tiles;
+                ++seg_no;
+                tg += seg_tiles;
+                cur.t += seg_tiles;
+                if (cur.t == cur.n_tiles) cur.next_pair(p);
+            }
+        }
+    } else if (warp < 8) {
+        if (TAIL) asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+        if (t_end > t_begin) {
+            // ================================================================ softmax / epilogue, rows 0..127
+            const int quarter = warp & 3;
+            const int r = quarter * 32 + lane;                 // row of the pair = TMEM lane
+            const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+            const uint32_t o_addr = tmem + lane_addr + O_COL0;
+            TileCursor cur;
+            cur.seek(p, start_b, start_prefix, t_begin, TILE);
+            uint32_t ug = 0;               // tiles of this block so far
+            uint32_t seg_no = 0;
+            bool ok = true;
+            for (long long tg = t_begin; tg < t_end && ok; ++seg_no) {
+                const int b = cur.b, g = cur.g;
+                const int seg_tiles = (int)min((long long)(cur.n_tiles - cur.t), t_end - tg);
+                const int R = cur.gam + 1, L = p.seq_len[b];
+                const int n_rows = G * R;
+                const bool warp_active = quarter * 32 < n_rows;
+                const bool row_ok = r < n_rows;
+                const int i = r / G, hh = r - i * G;
+                const int pos = L - R + i;                     // last visible key of this row
+                const long long q_row = ((long long)p.cu_q[b] + i) * p.hq + (long long)g * G + hh;
+                // ---- this thread's query row -> its tensor-memory lane (64 columns of bf16 pairs).
+                // Every tensor-core instruction that read the previous segment's rows has completed:
+                // this thread has seen the last S of that segment, and S follows all Q K^T in order.
+                if (warp_active) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(
+                        static_cast<const __nv_bfloat16 *>(p.q) + q_row * HD);
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf) {
+                        uint32_t qv[32];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const uint4 v = row_ok ? __ldg(src + hf * 8 + c) : make_uint4(0, 0, 0, 0);
+                            qv[4 * c] = v.x; qv[4 * c + 1] = v.y; qv[4 * c + 2] = v.z; qv[4 * c + 3] = v.w;
+                        }
+                        tc_st32(tmem + lane_addr + Q_COL0 + hf * 32, qv);
+                    }
+                    tc_wait_st();
+                    tc_fence_before();
+                }
+                mbar_arrive(smem_u32(&sh->q_full));
+                float m_ref = -CUDART_INF_F, l_sum = 0.f;
+                for (int ti = 0; ti < seg_tiles && ok; ++ti) {
+                    const uint32_t gu = ug + ti;
+                    const uint32_t s_addr = tmem + lane_addr + S_COL0 + (gu & 1) * TILE;
+                    ok = bounded_wait(smem_u32(&sh->s_full[gu & 1]), (gu >> 1) & 1, abort_flag, p.device_status);
+                    if (!ok) break;
+                    if (!warp_active) {                         // all 32 rows are padding
+                        mbar_arrive(smem_u32(&sh->p_full[gu & 1]));
+                        continue;
+                    }
+                    tc_fence_after();
+                    const int tok0 = (cur.t + ti) * TILE;
+                    const bool need_mask = tok0 + TILE - 1 > L - R;    // some row cannot see the whole tile
+                    uint32_t s[TILE];
+#pragma unroll
+                    for (int ch = 0; ch < TILE / 32; ++ch) tc_ld32_nowait(s_addr + ch * 32, s + ch * 32);
+                    tc_wait_ld();
+                    if (need_mask) {
+#pragma unroll
+                        for (int c = 0; c < TILE; ++c)
+                            if (tok0 + c > pos) s[c] = 0xff800000u;     // -inf
+                    }
+                    float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
+#pragma unroll
+                    for (int c = 0; c < TILE; c += 4) {
+                        m0 = fmaxf(m0, __uint_as_float(s[c]));
+                        m1 = fmaxf(m1, __uint_as_float(s[c + 1]));
+                        m2 = fmaxf(m2, __uint_as_float(s[c + 2]));
+                        m3 = fmaxf(m3, __uint_as_float(s[c + 3]));
+                    }
+                    const float m_tile = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * c_scale;
+                    float factor = 1.f;
+                    bool rescale = false;
+                    if (m_tile > m_ref + RESCALE_THRESHOLD || m_ref == -CUDART_INF_F) {
+                        if (m_tile > -CUDART_INF_F) {
+                            rescale = (m_ref > -CUDART_INF_F);
+                            factor = rescale ? ex2_approx(m_ref - m_tile) : 1.f;
+                            m_ref = m_tile;
+                        }
+                    }
+                    const float m_use = (m_ref == -CUDART_INF_F) ? 0.f : m_ref;
+                    if (rescale) l_sum *= factor;
+                    // tensor-memory accesses are warp-wide: if any row of the warp has to rescale
+                    // its accumulator, the whole warp goes through (factor 1 elsewhere)
+                    if (__any_sync(0xffffffffu, rescale && ti > 0)) {
+                        // the accumulator may only be touched once the previous PV is complete
+                        ok = bounded_wait(smem_u32(&sh->o_done[(gu - 1) & 1]), ((gu - 1) >> 1) & 1, abort_flag,
+                                          p.device_status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const float f = (rescale && ti > 0) ? factor : 1.f;
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            uint32_t o[32];
+                            tc_ld32(o_addr + ch * 32, o);
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
+                            tc_st32(o_addr + ch * 32, o);
+                        }
+                    }
+                    // P = 2^(s*c - m_ref) as bf16 pairs, written over S (masked scores are -inf -> 0)
+                    float tile_sum = 0.f;
+#pragma unroll
+                    for (int ch = 0; ch < TILE / 32; ++ch) {
+                        float sum0 = 0.f, sum1 = 0.f;
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int c = 0; c < 32; c += 2) {
+                            const float e0 = ex2_approx(fmaf(__uint_as_float(s[ch * 32 + c]), c_scale, -m_use));
+                            const float e1 = ex2_approx(fmaf(__uint_as_float(s[ch * 32 + c + 1]), c_scale, -m_use));
+                            sum0 += e0;
+                            sum1 += e1;
+                            pk[c >> 1] = pack_bf16(e0, e1);
+                        }
+                        tile_sum += sum0 + sum1;
+                        asm volatile(
+                            "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+                            "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(
+                                s_addr + ch * 16),
+                            "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]),
+                            "r"(pk[7]), "r"(pk[8]), "r"(pk[9]), "r"(pk[10]), "r"(pk[11]), "r"(pk[12]),
+                            "r"(pk[13]), "r"(pk[14]), "r"(pk[15])
+                            : "memory");
+                    }
+                    l_sum += tile_sum;
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&sh->p_full[gu & 1]));
+                }
+                if (!ok) break;
+                // ---- epilogue of the segment: wait for the last PV, then read O
+                {
+                    const uint32_t gl = ug + seg_tiles - 1;
+                    if (warp_active)
+                        ok = bounded_wait(smem_u32(&sh->o_done[gl & 1]), (gl >> 1) & 1, abort_flag, p.device_status);
+                }
+                if (!ok) break;
+                tc_fence_after();
+                const bool whole = (cur.t == 0 && seg_tiles == cur.n_tiles);
+                if (!warp_active) {
+                    // padding rows: nothing to write
+                } else if (whole) {
+                    const float inv = 1.f / l_sum;
+                    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.o) + q_row * HD;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t o[32];
+                        tc_ld32(o_addr + ch * 32, o);
+                        if (row_ok) {
+#pragma unroll
+                            for (int c = 0; c < 32; c += 8) {
+                                uint4 w;
+                                w.x = pack_bf16(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
+                                w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+                                w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+                                w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+                                *reinterpret_cast<uint4 *>(dst + ch * 32 + c) = w;
+                            }
+                        }
+                    }
+                    if (row_ok && p.lse != nullptr)
+                        p.lse[q_row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+                } else {
+                    // partial: fp32 O row, then max and sum; slot 0 = the block's first segment
+                    float *slot = a.ws_part + ((size_t)blockIdx.x * 2 + (seg_no == 0 ? 0 : 1)) * part_slot_floats(a.slot_rows);
+                    float *orow = slot + (size_t)r * HD;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t o[32];
+                        tc_ld32(o_addr + ch * 32, o);
+                        if (row_ok) {
+#pragma unroll
+                            for (int c = 0; c < 32; c += 4)
+                                *reinterpret_cast<uint4 *>(orow + ch * 32 + c) = make_uint4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+                        }
+                    }
+                    if (row_ok) {
+                        slot[(size_t)a.slot_rows * HD + r] = m_ref;
+                        slot[(size_t)a.slot_rows * HD + a.slot_rows + r] = l_sum;
+                    }
+                }
+                tc_fence_before();
+                ug += seg_tiles;
+                tg += seg_tiles;
+                cur.t += seg_tiles;
+                if (cur.t == cur.n_tiles) cur.next_pair(p);
+            }
+        }
+    } else {
+        if (TAIL) asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+        if (TAIL && t_end > t_begin) {
+            // ================================================================ tail rows 128..143
+            // Warp tw owns tokens [32 tw, 32 tw + 32) of every tile.  Fragment coordinates of
+            // mma.sync m16n8k16: g8 = row (and row + 8), t4 = column pair.
+            const int tw = warp - 8;
+            const int g8 = lane >> 2, t4 = lane & 3;
+            const int mi = lane >> 3, r8 = lane & 7;           // ldmatrix: matrix and row this lane addresses
+            TileCursor cur;
+            cur.seek(p, start_b, start_prefix, t_begin, TILE);
+            uint32_t ug = 0, seg_no = 0, sync_no = 0;
+            bool ok = true;
+            for (long long tg = t_begin; tg < t_end && ok; ++seg_no) {
+                const int b = cur.b, g = cur.g;
+                const int seg_tiles = (int)min((long long)(cur.n_tiles - cur.t), t_end - tg);
+                const int R = cur.gam + 1, L = p.seq_len[b];
+                const int n_rows = G * R;
+                const bool active = n_rows > 128;               // the pair has tail rows
+                int pos[2];
+                long long q_row[2];
+                bool row_ok[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int r = 128 + g8 + 8 * h;
+                    const int i = r / G, hh = r - i * G;
+                    row_ok[h] = r < n_rows;
+                    pos[h] = L - R + i;
+                    q_row[h] = ((long long)p.cu_q[b] + i) * p.hq + (long long)g * G + hh;
+                }
+                // A fragments of the 16 tail rows, all 8 k-steps of 16 dims (padding rows are zero)
+                uint32_t qa[8][4];
+                if (active) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t *src = reinterpret_cast<const uint32_t *>(
+                            static_cast<const __nv_bfloat16 *>(p.q) + q_row[h] * HD);
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            qa[ks][h] = row_ok[h] ? __ldg(src + ks * 8 + t4) : 0u;
+                            qa[ks][2 + h] = row_ok[h] ? __ldg(src + ks * 8 + 4 + t4) : 0u;
+                        }
+                    }
+                }
+                float m_ref[2] = {-CUDART_INF_F, -CUDART_INF_F}, l_sum[2] = {0.f, 0.f};
+                float o[16][4];
+#pragma unroll
+                for (int nd = 0; nd < 16; ++nd) o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f;
+
+                for (int ti = 0; ti < seg_tiles && ok; ++ti) {
+                    const uint32_t gu = ug + ti;
+                    const uint32_t item_k = 2 * gu, item_v = 2 * gu + 1;
+                    const uint32_t slot_k = item_k % (uint32_t)n_slots, slot_v = item_v % (uint32_t)n_slots;
+                    const int tok0 = (cur.t + ti) * TILE + tw * 32;       // first token of this warp's share
+                    const bool work = active && tok0 < L;                  // otherwise nothing visible
+                    ok = bounded_wait(smem_u32(&sh->full[slot_k]), (item_k / n_slots) & 1, abort_flag, p.device_status);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    uint32_t pa[2][4];
+                    if (work) {
+                        // ---- S (16 x 32) = Q K^T over 128 dims
+                        float sacc[4][4];
+                        const uint32_t kbase = smem_u32(ring + slot_k * SLOT_BYTES);
+#pragma unroll
+                        for (int nb = 0; nb < 4; ++nb) sacc[nb][0] = sacc[nb][1] = sacc[nb][2] = sacc[nb][3] = 0.f;
+                        // k-steps outside, token blocks inside: four independent accumulator chains
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) {
+                            const int c = 4 * kk + mi;                    // 16-byte chunk (8 dims) of the row
+#pragma unroll
+                            for (int nb = 0; nb < 4; ++nb) {
+                                const int token = tw * 32 + nb * 8 + r8;  // row of the tile this lane addresses
+                                const uint32_t addr = kbase + (c >> 3) * (SLOT_BYTES / 2) + token * 128 +
+                                                      (((c & 7) ^ (token & 7)) << 4);
+                                uint32_t b0, b1, b2, b3;
+                                ldmatrix_x4(addr, b0, b1, b2, b3);
+                                mma_16816(sacc[nb], qa[2 * kk], b0, b1);
+                                mma_16816(sacc[nb], qa[2 * kk + 1], b2, b3);
+                            }
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&sh->empty[slot_k]));
+                        // ---- online softmax of rows g8 (h = 0) and g8 + 8 (h = 1)
+                        float f[2] = {1.f, 1.f};
+                        bool resc = false;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            float mt = -CUDART_INF_F;
+#pragma unroll
+                            for (int nb = 0; nb < 4; ++nb)
+#pragma unroll
+                                for (int e = 0; e < 2; ++e) {
+                                    float x = sacc[nb][2 * h + e] * c_scale;
+                                    if (tok0 + nb * 8 + 2 * t4 + e > pos[h]) x = -CUDART_INF_F;
+                                    sacc[nb][2 * h + e] = x;
+                                    mt = fmaxf(mt, x);
+                                }
+                            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
+                            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
+                            if ((mt > m_ref[h] + RESCALE_THRESHOLD || m_ref[h] == -CUDART_INF_F) && mt > -CUDART_INF_F) {
+                                if (m_ref[h] > -CUDART_INF_F) {
+                                    f[h] = ex2_approx(m_ref[h] - mt);
+                                    resc = true;
+                                }
+                                m_ref[h] = mt;
+                            }
+                        }
+                        if (__any_sync(0xffffffffu, resc)) {
+                            l_sum[0] *= f[0];
+                            l_sum[1] *= f[1];
+#pragma unroll
+                            for (int nd = 0; nd < 16; ++nd) {
+                                o[nd][0] *= f[0]; o[nd][1] *= f[0];
+                                o[nd][2] *= f[1]; o[nd][3] *= f[1];
+                            }
+                        }
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const float m_use = (m_ref[h] == -CUDART_INF_F) ? 0.f : m_ref[h];
+                            float sum = 0.f;
+#pragma unroll
+                            for (int nb = 0; nb < 4; ++nb) {
+                                const float e0 = ex2_approx(sacc[nb][2 * h] - m_use);
+                                const float e1 = ex2_approx(sacc[nb][2 * h + 1] - m_use);
+                                sum += e0 + e1;
+                                // k-step j = nb / 2 of P V: registers h (tokens 0-7) and 2 + h (tokens 8-15)
+                                pa[nb >> 1][(nb & 1) * 2 + h] = pack_bf16(e0, e1);
+                            }
+                            l_sum[h] += sum;
+                        }
+                    } else {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&sh->empty[slot_k]));
+                    }
+                    ok = bounded_wait(smem_u32(&sh->full[slot_v]), (item_v / n_slots) & 1, abort_flag, p.device_status);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    if (work) {
+                        // ---- O (16 x 128) += P (16 x 32) V
+                        const uint32_t vbase = smem_u32(ring + slot_v * SLOT_BYTES);
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            const int token = tw * 32 + 16 * j + (mi & 1) * 8 + r8;
+#pragma unroll
+                            for (int nd2 = 0; nd2 < 8; ++nd2) {
+                                const int c = 2 * nd2 + (mi >> 1);
+                                const uint32_t addr = vbase + (c >> 3) * (SLOT_BYTES / 2) + token * 128 +
+                                                      (((c & 7) ^ (token & 7)) << 4);
+                                uint32_t b0, b1, b2, b3;
+                                ldmatrix_x4_trans(addr, b0, b1, b2, b3);
+                                mma_16816(o[2 * nd2], pa[j], b0, b1);
+                                mma_16816(o[2 * nd2 + 1], pa[j], b2, b3);
+                            }
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh->empty[slot_v]));
+                }
+                if (!ok) break;
+                // ---- merge the four warps' partial states through shared memory
+                if (active) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        l_sum[h] += __shfl_xor_sync(0xffffffffu, l_sum[h], 1);
+                        l_sum[h] += __shfl_xor_sync(0xffffffffu, l_sum[h], 2);
+                        const int row = g8 + 8 * h;
+#pragma unroll
+                        for (int nd = 0; nd < 16; ++nd)
+                            *reinterpret_cast<float2 *>(&tm->o[tw][row][nd * 8 + 2 * t4]) =
+                                make_float2(o[nd][2 * h], o[nd][2 * h + 1]);
+                        if (t4 == 0) {
+                            tm->m[tw][row] = m_ref[h];
+                            tm->l[tw][row] = l_sum[h];
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh->tail_sync));
+                    ok = bounded_wait(smem_u32(&sh->tail_sync), sync_no & 1, abort_flag, p.device_status);
+                    ++sync_no;
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    // thread j of the 128: row j / 8, dims 16 (j % 8) .. + 16
+                    const int j = tid - 256;
+                    const int row = j >> 3, d0 = (j & 7) * 16;
+                    const int r = 128 + row;
+                    if (r < n_rows) {
+                        float M = -CUDART_INF_F;
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) M = fmaxf(M, tm->m[w][row]);
+                        float acc[16];
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) acc[c] = 0.f;
+                        float lsum = 0.f;
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) {
+                            const float mw = tm->m[w][row];
+                            if (mw == -CUDART_INF_F) continue;
+                            const float sc = exp2f(mw - M);
+                            lsum += sc * tm->l[w][row];
+#pragma unroll
+                            for (int c = 0; c < 16; c += 4) {
+                                const float4 v = *reinterpret_cast<const float4 *>(&tm->o[w][row][d0 + c]);
+                                acc[c] += sc * v.x; acc[c + 1] += sc * v.y; acc[c + 2] += sc * v.z; acc[c + 3] += sc * v.w;
+                            }
+                        }
+                        const int i = r / G, hh = r - i * G;
+                        const long long qr = ((long long)p.cu_q[b] + i) * p.hq + (long long)g * G + hh;
+                        const bool whole = (cur.t == 0 && seg_tiles == cur.n_tiles);
+                        if (whole) {
+                            const float inv = 1.f / lsum;
+                            __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.o) + qr * HD + d0;
+#pragma unroll
+                            for (int c = 0; c < 16; c += 8) {
+                                uint4 w4;
+                                w4.x = pack_bf16(acc[c] * inv, acc[c + 1] * inv);
+                                w4.y = pack_bf16(acc[c + 2] * inv, acc[c + 3] * inv);
+                                w4.z = pack_bf16(acc[c + 4] * inv, acc[c + 5] * inv);
+                                w4.w = pack_bf16(acc[c + 6] * inv, acc[c + 7] * inv);
+                                *reinterpret_cast<uint4 *>(dst + c) = w4;
+                            }
+                            if ((j & 7) == 0 && p.lse != nullptr) p.lse[qr] = (M + log2f(lsum)) * 0.6931471805599453f;
+                        } else {
+                            float *slot = a.ws_part + ((size_t)blockIdx.x * 2 + (seg_no == 0 ? 0 : 1)) * part_slot_floats(a.slot_rows);
+                            float *orow = slot + (size_t)r * HD + d0;
+#pragma unroll
+                            for (int c = 0; c < 16; c += 4)
+                                *reinterpret_cast<float4 *>(orow + c) = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
+                            if ((j & 7) == 0) {
+                                slot[(size_t)a.slot_rows * HD + r] = M;
+                                slot[(size_t)a.slot_rows * HD + a.slot_rows + r] = lsum;
+                            }
+                        }
+                    }
+                    // the buffers are rewritten at the next segment's end: everyone must be done reading
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh->tail_sync));
+                    ok = bounded_wait(smem_u32(&sh->tail_sync), sync_no & 1, abort_flag, p.device_status);
+                    ++sync_no;
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
+                ug += seg_tiles;
+                tg += seg_tiles;
+                cur.t += seg_tiles;
+                if (cur.t == cur.n_tiles) cur.next_pair(p);
+            }
+        }
+    }
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------- host side
+bool attn_tq_supported(const sv_attn_params &p)
+{
+    if (p.head_dim != HD || p.pool == nullptr || !p.pool->has_maps) return false;
+    if (p.batch > MAX_BATCH_TC) return false;
+    const int rows = (p.hq / p.hkv) * (p.gamma_max + 1);
+    return rows >= 1 && rows <= 128 + TAIL_ROWS;
+}
+
+int attn_tq_slot_rows(int rows) { return rows > 128 ? 128 + TAIL_ROWS : 128; }
+
+template <bool TAIL>
+static sv_status launch_tq(AttnTcLaunch &a, const sv_attn_params &p, int grid, cudaStream_t stream)
+{
+    const size_t budget = 227 * 1024;
+    const size_t fixed = (TAIL ? sizeof(TailMerge) : 0) + ((sizeof(Shared) + 127) & ~(size_t)127);
+    a.n_slots = (int)((budget - fixed) / SLOT_BYTES);
+    if (a.n_slots > 8) a.n_slots = 8;
+    if (a.n_slots < 4) return SV_EUNSUPPORTED;
+    const size_t smem = fixed + (size_t)a.n_slots * SLOT_BYTES;
+    if (cudaFuncSetAttribute(attn_tq_kernel<TAIL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+        return SV_ECUDA;
+    attn_tq_kernel<TAIL><<<grid, TAIL ? 384 : 256, smem, stream>>>(a, p.pool->k_map, p.pool->v_map);
+    return launch_check();
+}
+
+sv_status launch_attn_tq_main(AttnTcLaunch &a, const sv_attn_params &p, int grid, cudaStream_t stream)
+{
+    return a.slot_rows > 128 ? launch_tq<true>(a, p, grid, stream) : launch_tq<false>(a, p, grid, stream);
+}
+
+}  // namespace sv
