@@ -83,6 +83,13 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4],
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// transpose of an 8x8 matrix of 16-bit elements held one row (4 x 2 elements) per 4 lanes
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x)
+{
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
@@ -93,11 +100,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 
 using namespace tq;
 
-template <bool TAIL>
-__global__ void __launch_bounds__(TAIL ? 384 : 256, 1)
+template <int NB>      // blocks of 8 tail rows beyond row 127 (0: no tail warps)
+__global__ void __launch_bounds__(NB > 0 ? 384 : 256, 1)
 attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                const __grid_constant__ CUtensorMap v_map)
 {
+    constexpr bool TAIL = NB > 0;
+    constexpr int NBA = NB > 0 ? NB : 1;               // array extent (no zero-length arrays)
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // carve: [ring slots][tail merge buffers][Shared]; the swizzled tiles need a 1024-byte aligned base
     uint8_t *ring = smem_raw;
@@ -193,9 +202,9 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
     int *abort_flag = &sh->abort_flag;
 
     // With the tail warps there are 384 threads and 168 registers each at launch; the producer /
-    // MMA warpgroup hands most of its share to the others (128 * (80 + 208 + 216) = 384 * 168).
+    // MMA warpgroup hands most of its share to the others (128 * (64 + 240 + 200) = 384 * 168).
     if (warp < 4) {
-        if (TAIL) asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+        if (TAIL) asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
         if (t_end > t_begin && warp != 1) {
             // ================================================================ TMA producers
             // One thread gets a tensor copy under way every ~90 cycles, and a tile needs 32 of
@@ -303,7 +312,7 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
             }
         }
     } else if (warp < 8) {
-        if (TAIL) asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+        if (TAIL) asm volatile("setmaxnreg.inc.sync.aligned.u32 240;");
         if (t_end > t_begin) {
             // ================================================================ softmax / epilogue, rows 0..127
             const int quarter = warp & 3;
@@ -494,11 +503,11 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
             }
         }
     } else {
-        if (TAIL) asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+        if (TAIL) asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
         if (TAIL && t_end > t_begin) {
             // ================================================================ tail rows 128..143
             // Warp tw owns tokens [32 tw, 32 tw + 32) of every tile.  Fragment coordinates of
-            // mma.sync m16n8k16: g8 = row (and row + 8), t4 = column pair.
+            // mma.sync m16n8k16: g8 = lane / 4, t4 = lane % 4.
             const int tw = warp - 8;
             const int g8 = lane >> 2, t4 = lane & 3;
             const int mi = lane >> 3, r8 = lane & 7;           // ldmatrix: matrix and row this lane addresses
@@ -512,35 +521,37 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 const int R = cur.gam + 1, L = p.seq_len[b];
                 const int n_rows = G * R;
                 const bool active = n_rows > 128;               // the pair has tail rows
-                int pos[2];
-                long long q_row[2];
-                bool row_ok[2];
+                // Transposed products, so that the 8-wide N side of m16n8k16 carries the rows:
+                //   S^T (tokens x rows) = K (tokens x dims) Q^T,   O^T (dims x rows) = V^T (dims x tokens) P^T.
+                // This thread's rows in block nbk: 8 nbk + 2 t4 + e (accumulator columns) and
+                // 8 nbk + g8 (B operand column).
+                int pos[NBA][2];
+                uint32_t qb[NBA][8][2];                           // B fragments of Q^T: [block][k-step][low / high 8 dims]
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int r = 128 + g8 + 8 * h;
+                for (int nbk = 0; nbk < NBA; ++nbk) {
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) pos[nbk][e] = L - R + (128 + 8 * nbk + 2 * t4 + e) / G;
+                    const int r = 128 + 8 * nbk + g8;
                     const int i = r / G, hh = r - i * G;
-                    row_ok[h] = r < n_rows;
-                    pos[h] = L - R + i;
-                    q_row[h] = ((long long)p.cu_q[b] + i) * p.hq + (long long)g * G + hh;
-                }
-                // A fragments of the 16 tail rows, all 8 k-steps of 16 dims (padding rows are zero)
-                uint32_t qa[8][4];
-                if (active) {
+                    const bool row_ok = active && r < n_rows;
+                    const uint32_t *src = reinterpret_cast<const uint32_t *>(
+                        static_cast<const __nv_bfloat16 *>(p.q) +
+                        (((long long)p.cu_q[b] + i) * p.hq + (long long)g * G + hh) * HD);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const uint32_t *src = reinterpret_cast<const uint32_t *>(
-                            static_cast<const __nv_bfloat16 *>(p.q) + q_row[h] * HD);
-#pragma unroll
-                        for (int ks = 0; ks < 8; ++ks) {
-                            qa[ks][h] = row_ok[h] ? __ldg(src + ks * 8 + t4) : 0u;
-                            qa[ks][2 + h] = row_ok[h] ? __ldg(src + ks * 8 + 4 + t4) : 0u;
-                        }
+                    for (int ks = 0; ks < 8; ++ks) {
+                        qb[nbk][ks][0] = row_ok ? __ldg(src + ks * 8 + t4) : 0u;
+                        qb[nbk][ks][1] = row_ok ? __ldg(src + ks * 8 + 4 + t4) : 0u;
                     }
                 }
-                float m_ref[2] = {-CUDART_INF_F, -CUDART_INF_F}, l_sum[2] = {0.f, 0.f};
-                float o[16][4];
+                float m_ref[NBA][2], l_sum[NBA][2];
+                float o[8][NBA][4];                               // O^T: [16-dim block][row block][fragment]
 #pragma unroll
-                for (int nd = 0; nd < 16; ++nd) o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f;
+                for (int nbk = 0; nbk < NBA; ++nbk) {
+                    m_ref[nbk][0] = m_ref[nbk][1] = -CUDART_INF_F;
+                    l_sum[nbk][0] = l_sum[nbk][1] = 0.f;
+#pragma unroll
+                    for (int md = 0; md < 8; ++md) o[md][nbk][0] = o[md][nbk][1] = o[md][nbk][2] = o[md][nbk][3] = 0.f;
+                }
 
                 for (int ti = 0; ti < seg_tiles && ok; ++ti) {
                     const uint32_t gu = ug + ti;
@@ -551,77 +562,115 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     ok = bounded_wait(smem_u32(&sh->full[slot_k]), (item_k / n_slots) & 1, abort_flag, p.device_status);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
-                    uint32_t pa[2][4];
+                    uint32_t pb[2][NBA][2];                                  // B fragments of P^T: [k-step][block][token half]
                     if (work) {
-                        // ---- S (16 x 32) = Q K^T over 128 dims
-                        float sacc[4][4];
+                        // ---- S^T (32 tokens x rows) over 128 dims
+                        // two accumulators per (token block, row block), even / odd k-steps: short chains
+                        float sacc[2][NBA][4], sodd[2][NBA][4];
                         const uint32_t kbase = smem_u32(ring + slot_k * SLOT_BYTES);
 #pragma unroll
-                        for (int nb = 0; nb < 4; ++nb) sacc[nb][0] = sacc[nb][1] = sacc[nb][2] = sacc[nb][3] = 0.f;
-                        // k-steps outside, token blocks inside: four independent accumulator chains
+                        for (int mb = 0; mb < 2; ++mb)
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            const int c = 4 * kk + mi;                    // 16-byte chunk (8 dims) of the row
+                            for (int nbk = 0; nbk < NBA; ++nbk)
 #pragma unroll
-                            for (int nb = 0; nb < 4; ++nb) {
-                                const int token = tw * 32 + nb * 8 + r8;  // row of the tile this lane addresses
-                                const uint32_t addr = kbase + (c >> 3) * (SLOT_BYTES / 2) + token * 128 +
-                                                      (((c & 7) ^ (token & 7)) << 4);
-                                uint32_t b0, b1, b2, b3;
-                                ldmatrix_x4(addr, b0, b1, b2, b3);
-                                mma_16816(sacc[nb], qa[2 * kk], b0, b1);
-                                mma_16816(sacc[nb], qa[2 * kk + 1], b2, b3);
+                                for (int x = 0; x < 4; ++x) sacc[mb][nbk][x] = sodd[mb][nbk][x] = 0.f;
+                        // The loads of four k-steps are issued together, then their MMAs: the asm
+                        // statements keep program order, and a load followed at once by its MMA
+                        // would cost a full shared-memory latency each time.
+#pragma unroll
+                        for (int kq = 0; kq < 2; ++kq) {
+                            uint32_t ka[4][2][4];
+#pragma unroll
+                            for (int k4 = 0; k4 < 4; ++k4) {
+                                const int c = 2 * (4 * kq + k4) + (mi >> 1);      // 16-byte chunk (8 dims) of the row
+#pragma unroll
+                                for (int mb = 0; mb < 2; ++mb) {
+                                    const int token = tw * 32 + mb * 16 + (mi & 1) * 8 + r8;
+                                    const uint32_t addr = kbase + (c >> 3) * (SLOT_BYTES / 2) + token * 128 +
+                                                          (((c & 7) ^ (token & 7)) << 4);
+                                    ldmatrix_x4(addr, ka[k4][mb][0], ka[k4][mb][1], ka[k4][mb][2], ka[k4][mb][3]);
+                                }
+                            }
+#pragma unroll
+                            for (int k4 = 0; k4 < 4; ++k4) {
+                                const int ks = 4 * kq + k4;
+#pragma unroll
+                                for (int mb = 0; mb < 2; ++mb) {
+                                    if (ks & 1) {
+                                        mma_16816(sodd[mb][0], ka[k4][mb], qb[0][ks][0], qb[0][ks][1]);
+                                        if (NB > 1) mma_16816(sodd[mb][NBA - 1], ka[k4][mb], qb[NBA - 1][ks][0], qb[NBA - 1][ks][1]);
+                                    } else {
+                                        mma_16816(sacc[mb][0], ka[k4][mb], qb[0][ks][0], qb[0][ks][1]);
+                                        if (NB > 1) mma_16816(sacc[mb][NBA - 1], ka[k4][mb], qb[NBA - 1][ks][0], qb[NBA - 1][ks][1]);
+                                    }
+                                }
                             }
                         }
+#pragma unroll
+                        for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+                            for (int nbk = 0; nbk < NBA; ++nbk)
+#pragma unroll
+                                for (int x = 0; x < 4; ++x) sacc[mb][nbk][x] += sodd[mb][nbk][x];
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&sh->empty[slot_k]));
-                        // ---- online softmax of rows g8 (h = 0) and g8 + 8 (h = 1)
-                        float f[2] = {1.f, 1.f};
+                        // ---- online softmax; a row's 32 scores sit in the 8 lanes with the same t4
+                        float f[NBA][2];
                         bool resc = false;
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            float mt = -CUDART_INF_F;
+                        for (int nbk = 0; nbk < NBA; ++nbk)
 #pragma unroll
-                            for (int nb = 0; nb < 4; ++nb)
+                            for (int e = 0; e < 2; ++e) {
+                                f[nbk][e] = 1.f;
+                                float mt = -CUDART_INF_F;
 #pragma unroll
-                                for (int e = 0; e < 2; ++e) {
-                                    float x = sacc[nb][2 * h + e] * c_scale;
-                                    if (tok0 + nb * 8 + 2 * t4 + e > pos[h]) x = -CUDART_INF_F;
-                                    sacc[nb][2 * h + e] = x;
-                                    mt = fmaxf(mt, x);
+                                for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+                                    for (int th = 0; th < 2; ++th) {
+                                        float x = sacc[mb][nbk][2 * th + e] * c_scale;
+                                        if (tok0 + mb * 16 + th * 8 + g8 > pos[nbk][e]) x = -CUDART_INF_F;
+                                        sacc[mb][nbk][2 * th + e] = x;
+                                        mt = fmaxf(mt, x);
+                                    }
+                                mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 4));
+                                mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 8));
+                                mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 16));
+                                float &m = m_ref[nbk][e];
+                                if ((mt > m + RESCALE_THRESHOLD || m == -CUDART_INF_F) && mt > -CUDART_INF_F) {
+                                    if (m > -CUDART_INF_F) {
+                                        f[nbk][e] = ex2_approx(m - mt);
+                                        resc = true;
+                                    }
+                                    m = mt;
                                 }
-                            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
-                            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
-                            if ((mt > m_ref[h] + RESCALE_THRESHOLD || m_ref[h] == -CUDART_INF_F) && mt > -CUDART_INF_F) {
-                                if (m_ref[h] > -CUDART_INF_F) {
-                                    f[h] = ex2_approx(m_ref[h] - mt);
-                                    resc = true;
-                                }
-                                m_ref[h] = mt;
                             }
-                        }
                         if (__any_sync(0xffffffffu, resc)) {
-                            l_sum[0] *= f[0];
-                            l_sum[1] *= f[1];
 #pragma unroll
-                            for (int nd = 0; nd < 16; ++nd) {
-                                o[nd][0] *= f[0]; o[nd][1] *= f[0];
-                                o[nd][2] *= f[1]; o[nd][3] *= f[1];
+                            for (int nbk = 0; nbk < NBA; ++nbk) {
+                                l_sum[nbk][0] *= f[nbk][0];
+                                l_sum[nbk][1] *= f[nbk][1];
+#pragma unroll
+                                for (int md = 0; md < 8; ++md) {
+                                    o[md][nbk][0] *= f[nbk][0]; o[md][nbk][1] *= f[nbk][1];
+                                    o[md][nbk][2] *= f[nbk][0]; o[md][nbk][3] *= f[nbk][1];
+                                }
                             }
                         }
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            const float m_use = (m_ref[h] == -CUDART_INF_F) ? 0.f : m_ref[h];
-                            float sum = 0.f;
+                        for (int nbk = 0; nbk < NBA; ++nbk) {
+                            const float mu0 = (m_ref[nbk][0] == -CUDART_INF_F) ? 0.f : m_ref[nbk][0];
+                            const float mu1 = (m_ref[nbk][1] == -CUDART_INF_F) ? 0.f : m_ref[nbk][1];
 #pragma unroll
-                            for (int nb = 0; nb < 4; ++nb) {
-                                const float e0 = ex2_approx(sacc[nb][2 * h] - m_use);
-                                const float e1 = ex2_approx(sacc[nb][2 * h + 1] - m_use);
-                                sum += e0 + e1;
-                                // k-step j = nb / 2 of P V: registers h (tokens 0-7) and 2 + h (tokens 8-15)
-                                pa[nb >> 1][(nb & 1) * 2 + h] = pack_bf16(e0, e1);
-                            }
-                            l_sum[h] += sum;
+                            for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+                                for (int th = 0; th < 2; ++th) {
+                                    const float e0 = ex2_approx(sacc[mb][nbk][2 * th] - mu0);
+                                    const float e1 = ex2_approx(sacc[mb][nbk][2 * th + 1] - mu1);
+                                    l_sum[nbk][0] += e0;
+                                    l_sum[nbk][1] += e1;
+                                    // (token g8, rows 2 t4, 2 t4 + 1) -> (row g8, tokens 2 t4, 2 t4 + 1)
+                                    pb[mb][nbk][th] = movmatrix_trans(pack_bf16(e0, e1));
+                                }
                         }
                     } else {
                         __syncwarp();
@@ -631,20 +680,23 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     if (work) {
-                        // ---- O (16 x 128) += P (16 x 32) V
+                        // ---- O^T (128 dims x rows) += V^T (dims x 32 tokens) P^T
                         const uint32_t vbase = smem_u32(ring + slot_v * SLOT_BYTES);
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
-                            const int token = tw * 32 + 16 * j + (mi & 1) * 8 + r8;
+                            const int token = tw * 32 + 16 * j + (mi >> 1) * 8 + r8;
+                            uint32_t va[8][4];                             // all eight loads first, then the MMAs
 #pragma unroll
-                            for (int nd2 = 0; nd2 < 8; ++nd2) {
-                                const int c = 2 * nd2 + (mi >> 1);
+                            for (int md = 0; md < 8; ++md) {
+                                const int c = 2 * md + (mi & 1);
                                 const uint32_t addr = vbase + (c >> 3) * (SLOT_BYTES / 2) + token * 128 +
                                                       (((c & 7) ^ (token & 7)) << 4);
-                                uint32_t b0, b1, b2, b3;
-                                ldmatrix_x4_trans(addr, b0, b1, b2, b3);
-                                mma_16816(o[2 * nd2], pa[j], b0, b1);
-                                mma_16816(o[2 * nd2 + 1], pa[j], b2, b3);
+                                ldmatrix_x4_trans(addr, va[md][0], va[md][1], va[md][2], va[md][3]);
+                            }
+#pragma unroll
+                            for (int md = 0; md < 8; ++md) {
+                                mma_16816(o[md][0], va[md], pb[j][0][0], pb[j][0][1]);
+                                if (NB > 1) mma_16816(o[md][NBA - 1], va[md], pb[j][NBA - 1][0], pb[j][NBA - 1][1]);
                             }
                         }
                     }
@@ -655,19 +707,24 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 // ---- merge the four warps' partial states through shared memory
                 if (active) {
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        l_sum[h] += __shfl_xor_sync(0xffffffffu, l_sum[h], 1);
-                        l_sum[h] += __shfl_xor_sync(0xffffffffu, l_sum[h], 2);
-                        const int row = g8 + 8 * h;
+                    for (int nbk = 0; nbk < NBA; ++nbk)
 #pragma unroll
-                        for (int nd = 0; nd < 16; ++nd)
-                            *reinterpret_cast<float2 *>(&tm->o[tw][row][nd * 8 + 2 * t4]) =
-                                make_float2(o[nd][2 * h], o[nd][2 * h + 1]);
-                        if (t4 == 0) {
-                            tm->m[tw][row] = m_ref[h];
-                            tm->l[tw][row] = l_sum[h];
+                        for (int e = 0; e < 2; ++e) {
+                            float l = l_sum[nbk][e];
+                            l += __shfl_xor_sync(0xffffffffu, l, 4);
+                            l += __shfl_xor_sync(0xffffffffu, l, 8);
+                            l += __shfl_xor_sync(0xffffffffu, l, 16);
+                            const int row = 8 * nbk + 2 * t4 + e;
+#pragma unroll
+                            for (int md = 0; md < 8; ++md) {
+                                tm->o[tw][row][16 * md + g8] = o[md][nbk][e];
+                                tm->o[tw][row][16 * md + g8 + 8] = o[md][nbk][2 + e];
+                            }
+                            if (g8 == 0) {
+                                tm->m[tw][row] = m_ref[nbk][e];
+                                tm->l[tw][row] = l;
+                            }
                         }
-                    }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&sh->tail_sync));
                     ok = bounded_wait(smem_u32(&sh->tail_sync), sync_no & 1, abort_flag, p.device_status);
@@ -760,26 +817,32 @@ bool attn_tq_supported(const sv_attn_params &p)
 }
 
 int attn_tq_slot_rows(int rows) { return rows > 128 ? 128 + TAIL_ROWS : 128; }
+static int g_tail_blocks(int rows) { return rows <= 128 ? 0 : (rows - 128 + 7) / 8; }
 
-template <bool TAIL>
+template <int NB>
 static sv_status launch_tq(AttnTcLaunch &a, const sv_attn_params &p, int grid, cudaStream_t stream)
 {
+    constexpr bool TAIL = NB > 0;
     const size_t budget = 227 * 1024;
     const size_t fixed = (TAIL ? sizeof(TailMerge) : 0) + ((sizeof(Shared) + 127) & ~(size_t)127);
     a.n_slots = (int)((budget - fixed) / SLOT_BYTES);
     if (a.n_slots > 8) a.n_slots = 8;
     if (a.n_slots < 4) return SV_EUNSUPPORTED;
     const size_t smem = fixed + (size_t)a.n_slots * SLOT_BYTES;
-    if (cudaFuncSetAttribute(attn_tq_kernel<TAIL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+    if (cudaFuncSetAttribute(attn_tq_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
         return SV_ECUDA;
-    attn_tq_kernel<TAIL><<<grid, TAIL ? 384 : 256, smem, stream>>>(a, p.pool->k_map, p.pool->v_map);
+    attn_tq_kernel<NB><<<grid, TAIL ? 384 : 256, smem, stream>>>(a, p.pool->k_map, p.pool->v_map);
     return launch_check();
 }
 
 sv_status launch_attn_tq_main(AttnTcLaunch &a, const sv_attn_params &p, int grid, cudaStream_t stream)
 {
-    return a.slot_rows > 128 ? launch_tq<true>(a, p, grid, stream) : launch_tq<false>(a, p, grid, stream);
+    switch (g_tail_blocks(a.group * (p.gamma_max + 1))) {
+        case 0: return launch_tq<0>(a, p, grid, stream);
+        case 1: return launch_tq<1>(a, p, grid, stream);
+        default: return launch_tq<2>(a, p, grid, stream);
+    }
 }
 
 }  // namespace sv
