@@ -35,6 +35,12 @@ from paper_2504_00030_b200 import shard, synth  # noqa: E402
 METRIC = "verified tokens/sec (verify step: attention + accept/resample + gamma update)"
 UNIT = "tokens/s"
 GT = dict(eta=0.5, delta=2.0, gamma_min=1)
+# DRAM traffic of the attention main kernel per algorithmic byte, from one ncu capture
+# (dram__bytes_read.sum + dram__bytes_write.sum of attn_tq_kernel<1> on the c5 shapes at batch
+# 32: 1.0552 GB + 0.0175 GB for 1 056 358 400 algorithmic bytes).  The workload there was cut
+# down to keep the capture short; traffic grows with the KV bytes, so the full launch's figure
+# is this ratio times its algorithmic bytes.  Set to None whenever the kernel changes.
+NCU_ATTN_TRAFFIC_RATIO = 1.0155
 
 
 def measured_peaks():
@@ -350,7 +356,9 @@ def run_ours(args):
                      "frac_of_8tbs": (attn_bytes + acc_bytes) / (ms_step * 1e-3) / 8e12,
                      "frac_of_measured": (attn_bytes + acc_bytes) / (ms_step * 1e-3) / 1e9 / peak},
         "roofline": {"bound": "hbm", "kernel": "spec_verify_attn", "achieved": achieved, "peak": peak,
-                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None},
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": (None if NCU_ATTN_TRAFFIC_RATIO is None or cfg.name != "c5"
+                                 else NCU_ATTN_TRAFFIC_RATIO * attn_bytes)},
         "accept_roofline": {"bound": "hbm", "achieved": acc_bytes / (t_acc * 1e-3) / 1e9, "peak": peak,
                             "unit": "GB/s", "frac": acc_bytes / (t_acc * 1e-3) / 1e9 / peak},
         "e2e": {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
