@@ -511,11 +511,18 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
 
 // ---------------------------------------------------------------------------- combine kernel
 // One block per (sequence, kv head); merges the partials of pairs whose tiles were shared
-// by several blocks of the main kernel.  Warp = query row.
-__global__ void __launch_bounds__(256)
+// by several blocks of the main kernel.  Warp = query row; a row's partials (running max, sum,
+// fp32 O) are all requested before the first is used, so a row costs one memory round trip.
+constexpr int COMBINE_THREADS = 1024;
+constexpr int COMBINE_LIST = 64;      // partial slots merged per pass
+
+__global__ void __launch_bounds__(COMBINE_THREADS)
 attn_combine_kernel(const AttnTcLaunch a)
 {
     const sv_attn_params &p = a.p;
+    __shared__ int s_list[COMBINE_LIST];
+    __shared__ int s_n;
+    __shared__ long long s_next;
     const int b = blockIdx.x / p.hkv, g = blockIdx.x % p.hkv;
     const int slot_rows = a.slot_rows;
     const long long grid = a.ws_prefix[p.batch + 1];
@@ -532,40 +539,81 @@ attn_combine_kernel(const AttnTcLaunch a)
     int gam = p.gamma[b];
     gam = min(max(gam, 0), p.gamma_max);
     const int G = a.group, n_rows = G * (gam + 1);
-    // one warp per query row: the lanes cover head_dim as float4, so every access is a full line
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     const size_t m_off = (size_t)slot_rows * HD, l_off = m_off + (size_t)slot_rows;
-    for (int r = warp; r < n_rows; r += n_warps) {
-        float m = -CUDART_INF_F;
-        for (long long c = c_first; c <= c_last; ++c) {
-            if (share_begin(c + 1, total, grid) == share_begin(c, total, grid)) continue;   // empty share
-            const int which = (share_begin(c, total, grid) >= T0) ? 0 : 1;
-            const float *slot = a.ws_part + ((size_t)c * 2 + which) * part_slot_floats(slot_rows);
-            m = fmaxf(m, slot[m_off + r]);
+    const size_t slot_floats = part_slot_floats(slot_rows);
+
+    // A pair split over more blocks than the list holds is merged in passes: each pass leaves
+    // its result in the pass's first slot (only this block touches the pair's slots) and the
+    // next pass starts from there.
+    int carry = -1;
+    for (long long c0 = c_first; c0 <= c_last;) {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int n = 0;
+            if (carry >= 0) s_list[n++] = carry;
+            long long c = c0;
+            for (; c <= c_last && n < COMBINE_LIST; ++c) {
+                const long long lo = share_begin(c, total, grid);
+                if (share_begin(c + 1, total, grid) == lo) continue;
+                s_list[n++] = (int)(c * 2 + (lo >= T0 ? 0 : 1));
+            }
+            s_n = n;
+            s_next = c;
         }
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        float l = 0.f;
-        for (long long c = c_first; c <= c_last; ++c) {
-            if (share_begin(c + 1, total, grid) == share_begin(c, total, grid)) continue;
-            const int which = (share_begin(c, total, grid) >= T0) ? 0 : 1;
-            const float *slot = a.ws_part + ((size_t)c * 2 + which) * part_slot_floats(slot_rows);
-            const float mc = slot[m_off + r];
-            if (mc == -CUDART_INF_F) continue;
-            const float w = exp2f(mc - m);
-            l += w * slot[l_off + r];
-            const float4 v = reinterpret_cast<const float4 *>(slot + (size_t)r * HD)[lane];
-            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+        __syncthreads();
+        const int n = s_n;
+        c0 = s_next;
+        const bool last = c0 > c_last;
+        carry = s_list[0];
+        for (int r = warp; r < n_rows; r += n_warps) {
+            float m_run = -CUDART_INF_F, l_run = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int j0 = 0; j0 < n; j0 += 4) {
+                float mc[4], lc[4];
+                float4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const bool have = j0 + u < n;
+                    const float *slot = a.ws_part + (size_t)s_list[have ? j0 + u : 0] * slot_floats;
+                    mc[u] = have ? slot[m_off + r] : -CUDART_INF_F;
+                    lc[u] = have ? slot[l_off + r] : 0.f;
+                    v[u] = have ? reinterpret_cast<const float4 *>(slot + (size_t)r * HD)[lane]
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                float m_new = m_run;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) m_new = fmaxf(m_new, mc[u]);
+                if (m_new == -CUDART_INF_F) continue;
+                const float w_old = exp2f(m_run - m_new);          // 0 while nothing has been merged
+                acc.x *= w_old; acc.y *= w_old; acc.z *= w_old; acc.w *= w_old;
+                l_run *= w_old;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (mc[u] == -CUDART_INF_F) continue;
+                    const float w = exp2f(mc[u] - m_new);
+                    l_run += w * lc[u];
+                    acc.x += w * v[u].x; acc.y += w * v[u].y; acc.z += w * v[u].z; acc.w += w * v[u].w;
+                }
+                m_run = m_new;
+            }
+            if (!last) {
+                float *slot = a.ws_part + (size_t)carry * slot_floats;
+                reinterpret_cast<float4 *>(slot + (size_t)r * HD)[lane] = acc;
+                if (lane == 0) { slot[m_off + r] = m_run; slot[l_off + r] = l_run; }
+                continue;
+            }
+            const int i = r / G, hh = r - i * G;
+            const long long q_row = ((long long)p.cu_q[b] + i) * p.hq + (long long)g * G + hh;
+            const float inv = 1.f / l_run;
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+            const __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+            uint2 packed;
+            packed.x = *reinterpret_cast<const uint32_t *>(&lo);
+            packed.y = *reinterpret_cast<const uint32_t *>(&hi);
+            reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.o) + q_row * HD)[lane] = packed;
+            if (lane == 0 && p.lse != nullptr) p.lse[q_row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
         }
-        const int i = r / G, hh = r - i * G;
-        const long long q_row = ((long long)p.cu_q[b] + i) * p.hq + (long long)g * G + hh;
-        const float inv = 1.f / l;
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-        const __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-        uint2 packed;
-        packed.x = *reinterpret_cast<const uint32_t *>(&lo);
-        packed.y = *reinterpret_cast<const uint32_t *>(&hi);
-        reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.o) + q_row * HD)[lane] = packed;
-        if (lane == 0 && p.lse != nullptr) p.lse[q_row] = (m + log2f(l)) * 0.6931471805599453f;
     }
 }
 
@@ -652,7 +700,7 @@ sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t worksp
     if (use_tq) st = launch_attn_tq_main(a, p, grid, stream);
     else st = a.nq == 1 ? launch_main<1, 64>(a, p, grid, stream) : launch_main<2, 128>(a, p, grid, stream);
     if (st != SV_OK) return st;
-    attn_combine_kernel<<<p.batch * p.hkv, 256, 0, stream>>>(a);
+    attn_combine_kernel<<<p.batch * p.hkv, COMBINE_THREADS, 0, stream>>>(a);
     return launch_check();
 }
 
