@@ -1,6 +1,6 @@
 // Fused speculative-sampling acceptance over the vocabulary (paper Section 3).
 //
-// Four kernels per step, all on the caller's stream:
+// Three kernels per step, all on the caller's stream:
 //
 //  1. accept_rowstats_kernel -- the streaming pass and the only one that touches every
 //     logit.  Each (row, slice of the vocabulary) item is owned by ONE WARP: 128-bit
@@ -9,14 +9,19 @@
 //     exponentials summed four at a time into a float64 accumulator, and a warp-shuffle
 //     reduction at the end.  No block-level synchronisation at all.  Greedy sequences
 //     (T = 0) only track (max, lowest index) of their target rows.
-//  2. accept_decide_kernel -- one block per sequence: merges the slice statistics into
-//     ln Z per row (float64), evaluates ratio_i = min(1, p_i[x_i]/q_i[x_i]) against u_i in
-//     float64 for all positions in parallel, then takes the first rejection.
-//  3. accept_segsum_kernel -- float64 pass over the one or two rows the next token is
-//     drawn from (residual max(0, p_n - q_n) or the bonus row): sums per 128-token
-//     segment, the sign of p_k - q_k decided with the first-pass partition sums.
-//  4. accept_pick_kernel -- one warp per sequence: exact partition sums, inverse CDF over
-//     the segment sums, exact float64 resolution inside the chosen segment.
+//  2. accept_decide_kernel -- one warp per sequence: merges the slice statistics into ln Z
+//     per row (float64), evaluates ratio_i = min(1, p_i[x_i]/q_i[x_i]) against u_i in float64
+//     for all positions in parallel, then takes the first rejection.
+//  3. accept_sample_kernel -- several blocks per sequence: float64 pass over the one or two
+//     rows the next token is drawn from (residual max(0, p_n - q_n) or the bonus row), sums
+//     per 128-token segment, the sign of p_k - q_k decided with the first-pass partition
+//     sums.  The block that finishes a sequence last runs the inverse CDF over the segment
+//     sums and resolves the token exactly inside the chosen segment.
+//
+// (Letting the streaming kernel's warps take the decisions or the float64 pass as they
+// become possible was measured and is slower: code that a warp runs once in a while is
+// fetched through an instruction cache that the streaming loop owns, under a saturated
+// memory system -- the decision alone then costs more than the whole kernel 2 and 3.)
 #include "common.cuh"
 
 #include <math_constants.h>
@@ -27,9 +32,10 @@ constexpr int RS_THREADS = 256;   // rowstats block (8 independent warps)
 constexpr int RS_UNROLL = 8;      // float4 loads in flight per lane
 constexpr int SEG = 128;          // vocabulary elements per sampling segment (one warp, float4 per lane)
 constexpr int SEG_THREADS = 256;
-constexpr int MAX_SPLITS = 16;    // blocks per sequence in the segment-sum pass
+constexpr int MAX_SPLITS = 16;    // blocks per sequence in the sampling kernel
 constexpr int MIN_SLICE = 2048;
 constexpr int MAX_SLICE = 16384;
+constexpr int MAX_GAMMA = 64;
 constexpr float REF_INIT = -1.0e30f;
 
 struct __align__(16) RowPartial {
@@ -40,8 +46,8 @@ struct __align__(16) RowPartial {
     int32_t pad;
 };
 
-// what the decision kernel leaves for the sampling kernels, one per sequence
-struct __align__(16) SeqRecord {
+// what the decision leaves for the sampling pass
+struct SeqRecord {
     double sum_p_hat, sum_q_hat;  // first-pass sums of the sampled rows (at ref_p / ref_q)
     float ref_p, ref_q;
     int32_t n;                    // first rejection (gamma if none)
@@ -51,7 +57,8 @@ struct __align__(16) SeqRecord {
 struct AcceptLaunch {
     sv_accept_params p;
     RowPartial *partials;   // [batch * (2 gmax + 1) * n_slices]
-    SeqRecord *records;     // [batch]
+    SeqRecord *records;     // [batch] written by the decision, read by the sampling kernel
+    unsigned int *done;     // [batch] blocks of the sampling kernel that finished (cleared by the decision kernel)
     double *seg;            // [batch][3][n_seg]: positive-part sums of a, of b, all of a
     double *totals;         // [batch][MAX_SPLITS][2]
     int slice;              // elements per slice (multiple of 1024)
@@ -59,6 +66,16 @@ struct AcceptLaunch {
     int n_seg;
     int splits;
     int vec_ok;             // 128-bit loads legal for every row
+};
+
+// shared scratch of the decision
+struct DecideScratch {
+    double logz[2 * MAX_GAMMA + 1];    // ln Z per dense row (natural log, of exp(x/T))
+    double rsum[2 * MAX_GAMMA + 1];    // merged sum and reference of each dense row
+    double ratio[MAX_GAMMA];
+    float rref[2 * MAX_GAMMA + 1];
+    int amax_idx[MAX_GAMMA + 1];
+    unsigned char code[MAX_GAMMA];
 };
 
 __device__ __forceinline__ float seq_temperature(const sv_accept_params &p, int b)
@@ -97,27 +114,75 @@ __device__ __forceinline__ void merge_argmax(float &v, int &i, float v2, int i2)
     if (v2 > v || (v2 == v && i2 < i)) { v = v2; i = i2; }
 }
 
-// 2^y in float64 for y <= ~4 (anything below -1000, -inf or NaN gives 0): round to the nearest
-// integer, degree-11 Taylor polynomial of 2^f on [-1/2, 1/2] (error < 1e-14), exponent added
-// by hand.
-__device__ __forceinline__ double exp2_f64(double y)
+// 2^(j/128), j = 0..127, correctly rounded
+__device__ const double g_exp2_table[128] = {
+    1.0, 1.0054299011128027, 1.0108892860517005, 1.016378314910953,
+    1.0218971486541166, 1.0274459491187637, 1.0330248790212284, 1.0386341019613787,
+    1.0442737824274138, 1.0499440858006872, 1.0556451783605572, 1.061377227289262,
+    1.0671404006768237, 1.0729348675259756, 1.0787607977571199, 1.0846183622133092,
+    1.0905077326652577, 1.0964290818163769, 1.102382583307841, 1.1083684117236787,
+    1.1143867425958924, 1.1204377524096067, 1.1265216186082418, 1.1326385195987192,
+    1.1387886347566916, 1.1449721444318042, 1.1511892299529827, 1.1574400736337511,
+    1.1637248587775775, 1.1700437696832502, 1.1763969916502812, 1.182784710984341,
+    1.189207115002721, 1.1956643920398273, 1.202156731452703, 1.2086843236265816,
+    1.215247359980469, 1.2218460329727576, 1.22848053610687, 1.2351510639369334,
+    1.241857812073484, 1.2486009771892048, 1.255380757024691, 1.2621973503942507,
+    1.2690509571917332, 1.275941778396392, 1.2828700160787783, 1.2898358734066657,
+    1.2968395546510096, 1.3038812651919358, 1.3109612115247644, 1.318079601266064,
+    1.3252366431597413, 1.3324325470831615, 1.339667524053303, 1.3469417862329458,
+    1.3542555469368927, 1.3616090206382248, 1.3690024229745905, 1.3764359707545302,
+    1.383909881963832, 1.3914243757719262, 1.3989796725383112, 1.4065759938190154,
+    1.4142135623730951, 1.4218926021691656, 1.42961333839197, 1.4373759974489824,
+    1.4451808069770467, 1.4530279958490526, 1.460917794180647, 1.4688504333369818,
+    1.4768261459394993, 1.4848451658727524, 1.4929077282912648, 1.5010140696264256,
+    1.5091644275934228, 1.5173590411982147, 1.5255981507445384, 1.533881997840956,
+    1.5422108254079407, 1.550584877685, 1.559004400237837, 1.567469639965553,
+    1.5759808451078865, 1.5845382652524937, 1.593142151342267, 1.6017927556826934,
+    1.6104903319492543, 1.6192351351948637, 1.6280274218573478, 1.6368674497669644,
+    1.645755478153965, 1.6546917676561943, 1.6636765803267364, 1.6727101796415966,
+    1.681792830507429, 1.6909247992693053, 1.7001063537185235, 1.709337763100463,
+    1.718619298122478, 1.7279512309618377, 1.7373338352737062, 1.746767386199169,
+    1.7562521603732995, 1.7657884359332727, 1.7753764925265212, 1.785016611318935,
+    1.7947090750031072, 1.804454167806624, 1.8142521755003989, 1.8241033854070534,
+    1.8340080864093424, 1.843966568958626, 1.8539791250833855, 1.864046048397789,
+    1.8741676341103, 1.8843441790323345, 1.8945759815869656, 1.9048633418176741,
+    1.9152065613971474, 1.925605943636125, 1.9360617934922943, 1.9465744175792332,
+    1.9571441241754002, 1.9677712232331759, 1.978456026387951, 1.9891988469672663,
+};
+
+// 2^y in float64 for y <= ~4 (anything below -1000, -inf or NaN gives 0).  y is split into
+// k/128 + r with k = rint(128 y): 2^y = 2^(k >> 7) * table[k & 127] * 2^r, |r| <= 1/256, 2^r by
+// its degree-5 Taylor polynomial (truncation below 1e-18); the power of two goes straight
+// into the exponent field.  N values at once, each step taken for all of them before the
+// next, so that the N dependent chains overlap in the pipeline; no branches.  `tab` is a
+// shared-memory copy of g_exp2_table.
+template <int N>
+__device__ __forceinline__ void exp2_f64_n(const double (&y)[N], double (&out)[N], const double *tab)
 {
-    if (!(y > -1000.0)) return 0.0;
-    const double n = rint(y);
-    const double f = y - n;
-    double p = 4.44553827187081e-10;
-    p = fma(p, f, 7.054911620801121e-09);
-    p = fma(p, f, 1.0178086009239696e-07);
-    p = fma(p, f, 1.3215486790144305e-06);
-    p = fma(p, f, 1.5252733804059838e-05);
-    p = fma(p, f, 0.00015403530393381606);
-    p = fma(p, f, 0.0013333558146428441);
-    p = fma(p, f, 0.009618129107628477);
-    p = fma(p, f, 0.055504108664821576);
-    p = fma(p, f, 0.2402265069591007);
-    p = fma(p, f, 0.6931471805599453);
-    p = fma(p, f, 1.0);
-    return __hiloint2double(__double2hiint(p) + ((int)n << 20), __double2loint(p));
+    constexpr double MAGIC = 6755399441055744.0;      // 1.5 * 2^52: adding it rounds to an integer
+    double r[N], t[N], q[N];
+    int k[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        const double yc = (y[i] > -1000.0) ? y[i] : -1000.0;     // NaN and -inf take this branch too
+        const double m = fma(yc, 128.0, MAGIC);
+        k[i] = __double2loint(m);
+        r[i] = fma(m - MAGIC, -0.0078125, yc);
+        t[i] = tab[k[i] & 127];
+        q[i] = 0.0013333558146428441;
+    }
+    constexpr double C[5] = {0.009618129107628477, 0.055504108664821576, 0.2402265069591007,
+                             0.6931471805599453, 1.0};
+#pragma unroll
+    for (int c = 0; c < 5; ++c)
+#pragma unroll
+        for (int i = 0; i < N; ++i) q[i] = fma(q[i], r[i], C[c]);
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        const double v = q[i] * t[i];
+        const double s = __hiloint2double(__double2hiint(v) + ((k[i] >> 7) << 20), __double2loint(v));
+        out[i] = (y[i] > -1000.0) ? s : 0.0;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -126,7 +191,7 @@ __device__ __forceinline__ double exp2_f64(double y)
 // j > gmax is draft row j-gmax-1.  Rows a sequence does not have this step are skipped.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(RS_THREADS)
-accept_rowstats_kernel(AcceptLaunch a)
+accept_rowstats_kernel(const __grid_constant__ AcceptLaunch a)
 {
     const sv_accept_params &p = a.p;
     const int rows_per_seq = 2 * p.gamma_max + 1;
@@ -258,22 +323,28 @@ accept_rowstats_kernel(AcceptLaunch a)
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// Kernel 2: ln Z per row, ratios, first rejection.  One block per sequence.
-// ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128)
-accept_decide_kernel(AcceptLaunch a)
+// a slice record written by the streaming kernel
+__device__ __forceinline__ RowPartial load_partial(const RowPartial *q)
 {
-    const sv_accept_params &p = a.p;
-    __shared__ double s_logz[2 * 64 + 1];    // ln Z per dense row (natural log, of exp(x/T))
-    __shared__ double s_rsum[2 * 64 + 1];    // merged sum and reference of each dense row
-    __shared__ float s_rref[2 * 64 + 1];
-    __shared__ int s_amax_idx[64 + 1];
-    __shared__ double s_ratio[64];
-    __shared__ unsigned char s_code[64];
+    const int4 v = __ldcg(reinterpret_cast<const int4 *>(q));
+    const int4 w = __ldcg(reinterpret_cast<const int4 *>(q) + 1);
+    RowPartial r;
+    r.sum = __hiloint2double(v.y, v.x);
+    r.ref = __int_as_float(v.z);
+    r.amax = __int_as_float(v.w);
+    r.aidx = w.x;
+    r.pad = 0;
+    return r;
+}
 
-    const int b = blockIdx.x;
-    const int tid = threadIdx.x;
+// ---------------------------------------------------------------------------------------------
+// Decision of one sequence (one warp): ln Z per row, ratios, first rejection; the record for
+// the sampling kernel goes to *rec_out.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideScratch *sc, int lane, SeqRecord *rec_out)
+{
+    constexpr bool write = true;
+    const sv_accept_params &p = a.p;
     const int gmax = p.gamma_max;
     const int rows_per_seq = 2 * gmax + 1;
     const int g = seq_gamma(p, b);
@@ -287,47 +358,55 @@ accept_decide_kernel(AcceptLaunch a)
     int32_t *out = p.out_tokens + (long long)b * (gmax + 1);
 
     // ---- merge the slice statistics of every row this sequence has
-    for (int j = tid; j < rows_per_seq; j += blockDim.x) {
+    for (int j = lane; j < rows_per_seq; j += 32) {
         const bool is_target = j <= gmax;
         const int i = is_target ? j : j - gmax - 1;
         const bool have = is_target ? (i <= g) : (i < g && !greedy);
         if (!have) continue;
         const RowPartial *pp = a.partials + ((long long)b * rows_per_seq + j) * a.n_slices;
+        RowPartial first = load_partial(pp);
         if (greedy) {
-            float v = pp[0].amax;
-            int ix = pp[0].aidx;
-            for (int s = 1; s < a.n_slices; ++s) merge_argmax(v, ix, pp[s].amax, pp[s].aidx);
-            s_amax_idx[i] = ix;
+            float v = first.amax;
+            int ix = first.aidx;
+            for (int s = 1; s < a.n_slices; ++s) {
+                const RowPartial q = load_partial(pp + s);
+                merge_argmax(v, ix, q.amax, q.aidx);
+            }
+            sc->amax_idx[i] = ix;
         } else {
-            float ref = pp[0].ref;
-            double sum = pp[0].sum;
-            for (int s = 1; s < a.n_slices; ++s) merge_stats(ref, sum, pp[s].ref, pp[s].sum);
-            s_rref[j] = ref;
-            s_rsum[j] = sum;
+            float ref = first.ref;
+            double sum = first.sum;
+            for (int s = 1; s < a.n_slices; ++s) {
+                const RowPartial q = load_partial(pp + s);
+                merge_stats(ref, sum, q.ref, q.sum);
+            }
+            sc->rref[j] = ref;
+            sc->rsum[j] = sum;
             // ln sum exp(x/T) = (ref + log2(sum)) * ln 2
             const double lz = ((double)ref + log2(sum)) * 0.6931471805599453;
-            s_logz[j] = lz;
-            if (is_target) { if (p.logZ_p != nullptr) p.logZ_p[p.cu_q[b] + i] = lz; }
-            else           { if (p.logZ_q != nullptr) p.logZ_q[p.cu_d[b] + i] = lz; }
+            sc->logz[j] = lz;
+            if (is_target) { if (write && p.logZ_p != nullptr) p.logZ_p[p.cu_q[b] + i] = lz; }
+            else           { if (write && p.logZ_q != nullptr) p.logZ_q[p.cu_d[b] + i] = lz; }
         }
     }
-    for (int i = tid; i <= gmax; i += blockDim.x) out[i] = -1;
-    __syncthreads();
+    if (write)
+        for (int i = lane; i <= gmax; i += 32) out[i] = -1;
+    __syncwarp();
 
     // ---- ratio and decision of every draft position in parallel (float64) ...
-    for (int i = tid; i < g; i += blockDim.x) {
+    for (int i = lane; i < g; i += 32) {
         const int xi = x[i];
         double r = 0.0;
         int code;   // 0 reject, 1 accept, 2 non-finite partition function
         int flag = 0;
         if (xi < 0 || xi >= V) {
-            set_status(p.device_status, SV_DEV_BAD_TOKEN);
+            if (write) set_status(p.device_status, SV_DEV_BAD_TOKEN);
             code = 0;
         } else if (greedy) {
-            code = (s_amax_idx[i] == xi) ? 1 : 0;
+            code = (sc->amax_idx[i] == xi) ? 1 : 0;
             r = (double)code;
         } else {
-            const double lzp = s_logz[i], lzq = s_logz[gmax + 1 + i];
+            const double lzp = sc->logz[i], lzq = sc->logz[gmax + 1 + i];
             if (!(isfinite(lzp) && isfinite(lzq))) {
                 code = 2;
             } else {
@@ -340,30 +419,30 @@ accept_decide_kernel(AcceptLaunch a)
                 flag = fabs(u - r) < 1e-6;
             }
         }
-        s_ratio[i] = r;
-        s_code[i] = (unsigned char)(code | (flag << 2));
+        sc->ratio[i] = r;
+        sc->code[i] = (unsigned char)(code | (flag << 2));
     }
-    __syncthreads();
-    // ... then the first rejection, which is sequential by definition: one thread
-    if (tid == 0) {
+    __syncwarp();
+    // ... then the first rejection, which is sequential by definition: one lane
+    if (lane == 0) {
         int n = g, ok = 1;
         uint32_t flags = 0;
         for (int i = 0; i < g; ++i) {
-            const int code = s_code[i] & 3;
+            const int code = sc->code[i] & 3;
             if (code == 2) { ok = 0; n = i; break; }
-            flags += (s_code[i] >> 2) & 1;
-            if (p.ratio != nullptr) p.ratio[p.cu_d[b] + i] = s_ratio[i];
+            flags += (sc->code[i] >> 2) & 1;
+            if (write && p.ratio != nullptr) p.ratio[p.cu_d[b] + i] = sc->ratio[i];
             if (code == 0) { n = i; break; }
         }
-        if (p.ratio != nullptr)
+        if (write && p.ratio != nullptr)
             for (int i = n + 1; i < g; ++i) p.ratio[p.cu_d[b] + i] = CUDART_NAN;
-        if (!greedy && ok && !isfinite(s_logz[n])) ok = 0;
-        if (!ok) set_status(p.device_status, SV_DEV_NONFINITE);
-        if (flags != 0 && p.flag_count != nullptr) atomicAdd(p.flag_count, flags);
-        p.n_accepted[b] = ok ? n : 0;
-        if (ok) {
+        if (!greedy && ok && !isfinite(sc->logz[n])) ok = 0;
+        if (write && !ok) set_status(p.device_status, SV_DEV_NONFINITE);
+        if (write && flags != 0 && p.flag_count != nullptr) atomicAdd(p.flag_count, flags);
+        if (write) p.n_accepted[b] = ok ? n : 0;
+        if (write && ok) {
             for (int i = 0; i < n; ++i) out[i] = x[i];
-            if (greedy) out[n] = s_amax_idx[n];
+            if (greedy) out[n] = sc->amax_idx[n];
         }
         SeqRecord rec;
         rec.n = n;
@@ -371,15 +450,27 @@ accept_decide_kernel(AcceptLaunch a)
         rec.ref_p = rec.ref_q = 0.f;
         rec.sum_p_hat = rec.sum_q_hat = 1.0;
         if (rec.mode != 0) {
-            rec.ref_p = s_rref[n];
-            rec.sum_p_hat = s_rsum[n];
+            rec.ref_p = sc->rref[n];
+            rec.sum_p_hat = sc->rsum[n];
             if (rec.mode == 1) {
-                rec.ref_q = s_rref[gmax + 1 + n];
-                rec.sum_q_hat = s_rsum[gmax + 1 + n];
+                rec.ref_q = sc->rref[gmax + 1 + n];
+                rec.sum_q_hat = sc->rsum[gmax + 1 + n];
             }
         }
-        a.records[b] = rec;
+        *rec_out = rec;
     }
+    __syncwarp();
+}
+
+// Kernel 2: one warp per sequence takes the decision; it also clears the sequence's completion
+// counter for kernel 3.
+__global__ void __launch_bounds__(32)
+accept_decide_kernel(const __grid_constant__ AcceptLaunch a)
+{
+    __shared__ DecideScratch s_dec;
+    const int b = blockIdx.x;
+    if (threadIdx.x == 0) a.done[b] = 0u;
+    decide_seq(a, b, &s_dec, threadIdx.x, a.records + b);
 }
 
 // four consecutive logits starting at k0 (k0 % 4 == 0), -inf past the vocabulary
@@ -395,78 +486,11 @@ __device__ __forceinline__ void load4(const float *row, int k0, int V, bool vec,
 }
 
 // ---------------------------------------------------------------------------------------------
-// Kernel 3: float64 segment sums of the sampled row(s).  grid = batch * splits.
-//   a_k = 2^(t_k c - ref_p), b_k = 2^(d_k c - ref_q), c = log2(e)/T
-//   per segment: sum of a over {p_k > q_k}, sum of b over the same set, sum of all a
-//   per block: sum of all a and all b (the exact partition sums, up to 2^ref)
+// Inverse CDF of one sequence, one warp (after all blocks of the sequence have stored their sums).
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(SEG_THREADS)
-accept_segsum_kernel(AcceptLaunch a)
+__device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const SeqRecord &rec, int lane, const double *tab)
 {
     const sv_accept_params &p = a.p;
-    __shared__ double s_red[2 * (SEG_THREADS / 32)];
-    const int b = blockIdx.x / a.splits, sp = blockIdx.x % a.splits;
-    const SeqRecord rec = a.records[b];
-    if (rec.mode == 0) return;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const bool residual = rec.mode == 1;
-    const int V = p.vocab, n_seg = a.n_seg;
-    const double c = 1.4426950408889634 / (double)seq_temperature(p, b);
-    const float *trow = p.target_logits + ((long long)p.cu_q[b] + rec.n) * p.row_stride;
-    const float *drow = residual ? p.draft_logits + ((long long)p.cu_d[b] + rec.n) * p.row_stride : nullptr;
-    const bool vec = a.vec_ok != 0;
-    const double ref_p = (double)rec.ref_p, ref_q = (double)rec.ref_q;
-    // first-pass partition sums, good to ~1e-7: only used to decide the sign of p_k - q_k
-    const double inv_zp_hat = 1.0 / rec.sum_p_hat, inv_zq_hat = 1.0 / rec.sum_q_hat;
-    double *seg_ap = a.seg + (size_t)b * 3 * n_seg, *seg_bp = seg_ap + n_seg, *seg_a = seg_bp + n_seg;
-
-    const int per = (n_seg + a.splits - 1) / a.splits;
-    const int s_begin = sp * per, s_end = min(n_seg, s_begin + per);
-    double tot_a = 0.0, tot_b = 0.0;
-    for (int s = s_begin + warp; s < s_end; s += SEG_THREADS / 32) {
-        const int k0 = s * SEG + 4 * lane;
-        float xt[4], xd[4];
-        load4(trow, k0, V, vec, xt);
-        if (residual) load4(drow, k0, V, vec, xd);
-        double sa = 0.0, sap = 0.0, sbp = 0.0, sb = 0.0;
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const double ak = exp2_f64((double)xt[u] * c - ref_p);
-            sa += ak;
-            if (residual) {
-                const double bk = exp2_f64((double)xd[u] * c - ref_q);
-                sb += bk;
-                if (ak * inv_zp_hat > bk * inv_zq_hat) { sap += ak; sbp += bk; }
-            }
-        }
-        tot_a += sa;
-        tot_b += sb;
-        sa = warp_sum_f64(sa);
-        if (residual) { sap = warp_sum_f64(sap); sbp = warp_sum_f64(sbp); }
-        if (lane == 0) { seg_a[s] = sa; seg_ap[s] = sap; seg_bp[s] = sbp; }
-    }
-    tot_a = warp_sum_f64(tot_a);
-    tot_b = warp_sum_f64(tot_b);
-    if (lane == 0) { s_red[warp] = tot_a; s_red[SEG_THREADS / 32 + warp] = tot_b; }
-    __syncthreads();
-    if (tid == 0) {
-        double za = 0.0, zb = 0.0;
-        for (int w = 0; w < SEG_THREADS / 32; ++w) { za += s_red[w]; zb += s_red[SEG_THREADS / 32 + w]; }
-        a.totals[((size_t)b * MAX_SPLITS + sp) * 2] = za;
-        a.totals[((size_t)b * MAX_SPLITS + sp) * 2 + 1] = zb;
-    }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Kernel 4: inverse CDF.  One warp per sequence.
-// ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(32)
-accept_pick_kernel(AcceptLaunch a)
-{
-    const sv_accept_params &p = a.p;
-    const int b = blockIdx.x, lane = threadIdx.x;
-    const SeqRecord rec = a.records[b];
-    if (rec.mode == 0) return;
     const bool residual = rec.mode == 1;
     const int V = p.vocab, n_seg = a.n_seg, n = rec.n;
     const double c = 1.4426950408889634 / (double)seq_temperature(p, b);
@@ -478,8 +502,8 @@ accept_pick_kernel(AcceptLaunch a)
 
     double Zp = 0.0, Zq = 0.0;
     for (int sp = 0; sp < a.splits; ++sp) {
-        Zp += a.totals[((size_t)b * MAX_SPLITS + sp) * 2];
-        Zq += a.totals[((size_t)b * MAX_SPLITS + sp) * 2 + 1];
+        Zp += __ldcg(&a.totals[((size_t)b * MAX_SPLITS + sp) * 2]);
+        Zq += __ldcg(&a.totals[((size_t)b * MAX_SPLITS + sp) * 2 + 1]);
     }
     const double inv_zp = 1.0 / Zp, inv_zq = residual ? 1.0 / Zq : 0.0;
 
@@ -487,7 +511,7 @@ accept_pick_kernel(AcceptLaunch a)
     const int per = (n_seg + 31) / 32;
     const int s_lo = min(lane * per, n_seg), s_hi = min(s_lo + per, n_seg);
     auto seg_w = [&](int s, bool use_r) {
-        return use_r ? seg_ap[s] * inv_zp - seg_bp[s] * inv_zq : seg_a[s] * inv_zp;
+        return use_r ? __ldcg(&seg_ap[s]) * inv_zp - __ldcg(&seg_bp[s]) * inv_zq : __ldcg(&seg_a[s]) * inv_zp;
     };
     double mine = 0.0;
     if (residual) for (int s = s_lo; s < s_hi; ++s) mine += seg_w(s, true);
@@ -528,10 +552,17 @@ accept_pick_kernel(AcceptLaunch a)
         float xt[4], xd[4];
         load4(trow, k0, V, vec, xt);
         if (use_resid) load4(drow, k0, V, vec, xd);
+        double y[8], e[8];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const double pk = exp2_f64((double)xt[u] * c - ref_p) * inv_zp;
-            w[u] = use_resid ? fmax(pk - exp2_f64((double)xd[u] * c - ref_q) * inv_zq, 0.0) : pk;
+            y[u] = (double)xt[u] * c - ref_p;
+            y[4 + u] = use_resid ? (double)xd[u] * c - ref_q : -2000.0;
+        }
+        exp2_f64_n<8>(y, e, tab);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const double pk = e[u] * inv_zp;
+            w[u] = use_resid ? fmax(pk - e[4 + u] * inv_zq, 0.0) : pk;
         }
     };
 
@@ -587,6 +618,109 @@ accept_pick_kernel(AcceptLaunch a)
 }
 
 // ---------------------------------------------------------------------------------------------
+// Kernel 3: float64 segment sums of the sampled row(s), inverse CDF.
+// grid = batch * splits.
+//   a_k = 2^(t_k c - ref_p), b_k = 2^(d_k c - ref_q), c = log2(e)/T
+//   per segment: sum of a over {p_k > q_k}, sum of b over the same set, sum of all a
+//   per block: sum of all a and all b (the exact partition sums, up to 2^ref)
+// ---------------------------------------------------------------------------------------------
+// Four blocks (32 warps) per SM: the pass is a mix of float64 arithmetic and shuffles that no
+// pipe saturates, so throughput follows the number of resident warps; 64 registers suffice.
+__global__ void __launch_bounds__(SEG_THREADS, 4)
+accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
+{
+    const sv_accept_params &p = a.p;
+    __shared__ double s_tab[128];
+    __shared__ double s_red[2 * (SEG_THREADS / 32)];
+    __shared__ int s_last;
+    const int b = blockIdx.x / a.splits, sp = blockIdx.x % a.splits;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid >= 128) s_tab[tid - 128] = g_exp2_table[tid - 128];
+    __syncthreads();
+    const SeqRecord rec = a.records[b];
+    if (rec.mode == 0) return;                        // greedy, or the sequence failed: nothing to sample
+    const bool residual = rec.mode == 1;
+    const int V = p.vocab, n_seg = a.n_seg;
+    const double c = 1.4426950408889634 / (double)seq_temperature(p, b);
+    const float *trow = p.target_logits + ((long long)p.cu_q[b] + rec.n) * p.row_stride;
+    const float *drow = residual ? p.draft_logits + ((long long)p.cu_d[b] + rec.n) * p.row_stride : nullptr;
+    const bool vec = a.vec_ok != 0;
+    const double ref_p = (double)rec.ref_p, ref_q = (double)rec.ref_q;
+    // first-pass partition sums, good to ~1e-7: only used to decide the sign of p_k - q_k
+    const double inv_zp_hat = 1.0 / rec.sum_p_hat, inv_zq_hat = 1.0 / rec.sum_q_hat;
+    double *seg_ap = a.seg + (size_t)b * 3 * n_seg, *seg_bp = seg_ap + n_seg, *seg_a = seg_bp + n_seg;
+
+    const int per = (n_seg + a.splits - 1) / a.splits;
+    const int s_begin = sp * per, s_end = min(n_seg, s_begin + per);
+    double tot_a = 0.0, tot_b = 0.0;
+    constexpr int UN = 1;               // segments whose loads are issued together
+    constexpr int NW = SEG_THREADS / 32;
+    for (int s0 = s_begin + warp; s0 < s_end; s0 += UN * NW) {
+        float xt[UN][4], xd[UN][4];
+#pragma unroll
+        for (int q = 0; q < UN; ++q) {
+            const int s = s0 + q * NW;
+            if (s < s_end) {
+                load4(trow, s * SEG + 4 * lane, V, vec, xt[q]);
+                if (residual) load4(drow, s * SEG + 4 * lane, V, vec, xd[q]);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < UN; ++q) {
+            const int s = s0 + q * NW;
+            if (s >= s_end) break;
+            double sa = 0.0, sap = 0.0, sbp = 0.0, sb = 0.0;
+            if (residual) {
+                // the eight exponentials of this lane (four tokens, two rows) as overlapping chains
+                double y[8], w[8];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    y[u] = (double)xt[q][u] * c - ref_p;
+                    y[4 + u] = (double)xd[q][u] * c - ref_q;
+                }
+                exp2_f64_n<8>(y, w, s_tab);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const double ak = w[u], bk = w[4 + u];
+                    sa += ak;
+                    sb += bk;
+                    if (ak * inv_zp_hat > bk * inv_zq_hat) { sap += ak; sbp += bk; }
+                }
+            } else {
+                double y[4], w[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) y[u] = (double)xt[q][u] * c - ref_p;
+                exp2_f64_n<4>(y, w, s_tab);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) sa += w[u];
+            }
+            tot_a += sa;
+            tot_b += sb;
+            sa = warp_sum_f64(sa);
+            if (residual) { sap = warp_sum_f64(sap); sbp = warp_sum_f64(sbp); }
+            if (lane == 0) { seg_a[s] = sa; seg_ap[s] = sap; seg_bp[s] = sbp; }
+        }
+    }
+    tot_a = warp_sum_f64(tot_a);
+    tot_b = warp_sum_f64(tot_b);
+    if (lane == 0) { s_red[warp] = tot_a; s_red[NW + warp] = tot_b; }
+    __syncthreads();          // also orders every warp's segment stores before the counter below
+    if (tid == 0) {
+        double za = 0.0, zb = 0.0;
+        for (int w = 0; w < NW; ++w) { za += s_red[w]; zb += s_red[NW + w]; }
+        a.totals[((size_t)b * MAX_SPLITS + sp) * 2] = za;
+        a.totals[((size_t)b * MAX_SPLITS + sp) * 2 + 1] = zb;
+        __threadfence();
+        s_last = atomicAdd(&a.done[b], 1u) + 1 == (unsigned)a.splits;
+    }
+    __syncthreads();
+    if (s_last && warp == 0) {
+        __threadfence();
+        pick_seq(a, b, rec, lane, s_tab);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
 static int pick_slice(const sv_accept_params *p)
@@ -602,7 +736,7 @@ static int pick_slice(const sv_accept_params *p)
 static size_t align256(size_t n) { return (n + 255) & ~(size_t)255; }
 
 struct AcceptLayout {
-    size_t partials, records, seg, totals, total;
+    size_t partials, records, ctl, seg, totals, total;
 };
 
 static AcceptLayout accept_layout(int batch, int gamma_max, int vocab, int slice)
@@ -612,7 +746,8 @@ static AcceptLayout accept_layout(int batch, int gamma_max, int vocab, int slice
     const size_t n_seg = ((size_t)vocab + SEG - 1) / SEG;
     l.partials = 0;
     l.records = align256((size_t)batch * (2 * (size_t)gamma_max + 1) * n_slices * sizeof(RowPartial));
-    l.seg = l.records + align256((size_t)batch * sizeof(SeqRecord));
+    l.ctl = l.records + align256((size_t)batch * sizeof(SeqRecord));
+    l.seg = l.ctl + align256((size_t)batch * sizeof(unsigned int));
     l.totals = l.seg + align256((size_t)batch * 3 * n_seg * sizeof(double));
     l.total = l.totals + align256((size_t)batch * MAX_SPLITS * 2 * sizeof(double));
     return l;
@@ -621,7 +756,7 @@ static AcceptLayout accept_layout(int batch, int gamma_max, int vocab, int slice
 static sv_status check_accept(const sv_accept_params *p)
 {
     if (p == nullptr || p->batch <= 0 || p->vocab <= 0 || p->gamma_max < 0) return SV_EINVAL;
-    if (p->gamma_max > 64) return SV_EUNSUPPORTED;
+    if (p->gamma_max > MAX_GAMMA) return SV_EUNSUPPORTED;
     if (p->target_logits == nullptr || p->gamma == nullptr || p->cu_q == nullptr ||
         p->cu_d == nullptr || p->n_accepted == nullptr || p->out_tokens == nullptr)
         return SV_EINVAL;
@@ -634,7 +769,7 @@ static sv_status check_accept(const sv_accept_params *p)
     return SV_OK;
 }
 
-// the four launches; `scratch` holds accept_layout(..., slice).total bytes
+// the three launches; `scratch` holds accept_layout(..., slice).total bytes
 static sv_status launch_accept(const sv_accept_params *p, void *scratch, int slice, cudaStream_t stream)
 {
     const AcceptLayout l = accept_layout(p->batch, p->gamma_max, p->vocab, slice);
@@ -643,6 +778,7 @@ static sv_status launch_accept(const sv_accept_params *p, void *scratch, int sli
     a.p = *p;
     a.partials = reinterpret_cast<RowPartial *>(base + l.partials);
     a.records = reinterpret_cast<SeqRecord *>(base + l.records);
+    a.done = reinterpret_cast<unsigned int *>(base + l.ctl);
     a.seg = reinterpret_cast<double *>(base + l.seg);
     a.totals = reinterpret_cast<double *>(base + l.totals);
     a.slice = slice;
@@ -650,20 +786,14 @@ static sv_status launch_accept(const sv_accept_params *p, void *scratch, int sli
     a.n_seg = (p->vocab + SEG - 1) / SEG;
     a.vec_ok = (p->row_stride % 4 == 0) && aligned16(p->target_logits) &&
                (p->draft_logits == nullptr || aligned16(p->draft_logits));
-    // blocks per sequence in the float64 pass: fill the machine once (a second, nearly empty
-    // wave would double the time), at least 8 segments per block
-    static int seg_blocks_per_sm = 0;
-    if (seg_blocks_per_sm == 0) {
-        int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, accept_segsum_kernel, SEG_THREADS, 0) !=
-                cudaSuccess || n < 1)
-            n = 2;
-        seg_blocks_per_sm = n;
-    }
-    int splits = (seg_blocks_per_sm * sm_count()) / p->batch;
+    // blocks per sequence in the sampling kernel: the float64 pass is bound by arithmetic, so
+    // several small blocks per SM (about eight) balance better than one wave of large ones; at
+    // least 8 segments per block; one block when nothing samples
+    const bool any_sampling = p->temperature_per_seq != nullptr || p->temperature > 0.f;
+    int splits = (8 * sm_count() + p->batch - 1) / p->batch;
     if (splits > MAX_SPLITS) splits = MAX_SPLITS;
     if (splits > (a.n_seg + 7) / 8) splits = (a.n_seg + 7) / 8;
-    if (splits < 1) splits = 1;
+    if (splits < 1 || !any_sampling) splits = 1;
     a.splits = splits;
 
     const long long n_items = (long long)p->batch * (2 * p->gamma_max + 1) * a.n_slices;
@@ -680,15 +810,10 @@ static sv_status launch_accept(const sv_accept_params *p, void *scratch, int sli
     accept_rowstats_kernel<<<(int)(blocks_needed < cap ? blocks_needed : cap), RS_THREADS, 0, stream>>>(a);
     sv_status st = launch_check();
     if (st != SV_OK) return st;
-    accept_decide_kernel<<<p->batch, 128, 0, stream>>>(a);
+    accept_decide_kernel<<<p->batch, 32, 0, stream>>>(a);
     st = launch_check();
     if (st != SV_OK) return st;
-    const bool any_sampling = p->temperature_per_seq != nullptr || p->temperature > 0.f;
-    if (!any_sampling) return SV_OK;
-    accept_segsum_kernel<<<(unsigned)(splits * p->batch), SEG_THREADS, 0, stream>>>(a);
-    st = launch_check();
-    if (st != SV_OK) return st;
-    accept_pick_kernel<<<p->batch, 32, 0, stream>>>(a);
+    accept_sample_kernel<<<(unsigned)(splits * p->batch), SEG_THREADS, 0, stream>>>(a);
     return launch_check();
 }
 
