@@ -61,6 +61,34 @@ def test_config_c5_shape_reduced_batch():
     check_accept(li, cfg.temperature, g, cu_q, cu_d, cfg.gamma_max)
 
 
+def test_full_size_c5_sampled_sequences():
+    """The largest configuration at full size, launched as the benchmark launches it (batch 128,
+    gamma 16 for every sequence, fixed row slabs): 12 sampled sequences against the oracle."""
+    cfg = synth.scaled(synth.CONFIGS["c5"], gamma_lo=16, gamma_hi=16)
+    li, g, cu_q, cu_d = case(cfg, padded=True)
+    gpu = run_accept_gpu(li, cfg.temperature, g, cu_q, cu_d, cfg.gamma_max)
+    assert gpu.status == 0
+    pick = np.sort(np.random.default_rng(5).choice(cfg.batch, 12, replace=False))
+    q_rows = np.concatenate([np.arange(cu_q[b], cu_q[b + 1]) for b in pick])
+    d_rows = np.concatenate([np.arange(cu_d[b], cu_d[b + 1]) for b in pick])
+    sub = synth.LogitInputs(li.target_logits[q_rows], li.draft_logits[d_rows], li.draft_tokens[d_rows],
+                            li.u_accept[d_rows], li.u_sample[pick])
+    sub_q, sub_d = synth.padded_offsets(len(pick), cfg.gamma_max)
+    from tests.harness import AcceptOut
+    gpu_sub = AcceptOut(gpu.n_accepted[pick], gpu.out_tokens[pick], gpu.ratio[d_rows], gpu.logZ_p[q_rows],
+                        gpu.logZ_q[d_rows], 0, 0)
+    ref, _, _ = compare_accept(gpu_sub, sub, cfg.temperature, g[pick], sub_q, sub_d, cfg.gamma_max)
+    seen = np.isfinite(ref.logZ_p)            # rows the oracle evaluated (up to the first rejection)
+    assert seen.any() and np.abs(np.expm1(gpu_sub.logZ_p[seen] - ref.logZ_p[seen])).max() <= 1e-5
+    # properties that hold at any size: counts in range, accepted tokens are the drafts, one
+    # token follows them and padding after it
+    assert ((gpu.n_accepted >= 0) & (gpu.n_accepted <= g)).all()
+    for b in range(cfg.batch):
+        n = gpu.n_accepted[b]
+        assert np.array_equal(gpu.out_tokens[b, :n], li.draft_tokens[cu_d[b]:cu_d[b] + n])
+        assert 0 <= gpu.out_tokens[b, n] < cfg.vocab and (gpu.out_tokens[b, n + 1:] == -1).all()
+
+
 @pytest.mark.parametrize("V", [1, 2, 3, 5, 127, 129, 1001, 4099])
 def test_small_and_odd_vocabularies(V):
     # V < one warp segment, V % 4 != 0 (scalar loads, unaligned rows), ragged tails
