@@ -1,6 +1,10 @@
 // Work schedule shared by the tensor-core attention kernels: the key tiles of the whole batch
-// form one list (sequence-major, then kv head, then tile); every persistent block takes an equal
-// contiguous share of it.
+// form one list (sequence-major, then kv head, then tile); every persistent block takes a
+// contiguous share of it.  Shares are equal in COST, not in tiles: starting a (sequence, kv
+// head) pair -- new query rows, a drained pipeline, an epilogue -- was measured to cost as much
+// as a few tiles, so a pair counts as its tiles plus `seg_cost`; otherwise a block whose share
+// holds many short sequences finishes long after the others.  Block c writes the first tile of
+// its share to bounds[c] in the workspace, where the combine kernel finds it.
 #pragma once
 
 #include "attn_common.cuh"
@@ -17,7 +21,7 @@ struct AttnTcLaunch {
     int nq;              // row groups of 128 rows (1 or 2)
     int slot_rows;       // query rows per partial-result slot
     int n_slots;         // K/V ring slots
-    int32_t *ws_prefix;  // [batch+1] tile prefix, then [2]: total tiles, grid size
+    int32_t *ws_prefix;  // [batch+1] tile prefix (last = total), grid size, then bounds[grid+1]
     float *ws_part;      // partial results: slot-major
 };
 
@@ -29,6 +33,8 @@ __device__ __forceinline__ long long share_begin(long long c, long long total, l
 {
     return (c * total) / grid;
 }
+
+constexpr int MAX_ATTN_GRID = 1024;     // blocks of a main kernel (bounds table in the workspace)
 
 // Tiles and validated gamma of one sequence; sequences with inconsistent lengths own no tiles.
 __device__ __forceinline__ int seq_tiles(const sv_attn_params &p, int b, int *gam_out, bool report, int tile)
@@ -46,6 +52,106 @@ __device__ __forceinline__ int seq_tiles(const sv_attn_params &p, int b, int *ga
     }
     if (gam_out != nullptr) *gam_out = g;
     return nt;
+}
+
+// What a block learns in its prologue.
+struct BlockShare {
+    int total_tiles;             // tiles of all sequences, per kv head
+    long long t_begin, t_end;    // the block's tiles of the global list
+    int start_b, start_prefix;   // sequence that holds t_begin and the tiles (per kv head) before it
+};
+
+// Computes the calling block's share (whole warp); block 0 also publishes the tile prefix and
+// the grid size for the combine kernel, and every block its lower bound.
+__device__ __forceinline__ void plan_block_share(const AttnTcLaunch &a, int lane, int tile, int seg_cost,
+                                                 BlockShare &o)
+{
+    const sv_attn_params &p = a.p;
+    const int batch = p.batch, hkv = p.hkv;
+    int32_t *bounds = a.ws_prefix + batch + 2;
+    // pass 1: totals, real and with the per-pair cost added
+    int carry = 0, carry_v = 0;
+    if (blockIdx.x == 0 && lane == 0) a.ws_prefix[0] = 0;
+    for (int base = 0; base < batch; base += 32) {
+        const int b = base + lane;
+        const int nt = (b < batch) ? seq_tiles(p, b, nullptr, blockIdx.x == 0, tile) : 0;
+        int v = nt, vv = nt > 0 ? nt + seg_cost : 0;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, v, d), tv = __shfl_up_sync(0xffffffffu, vv, d);
+            if (lane >= d) { v += t; vv += tv; }
+        }
+        if (blockIdx.x == 0 && b < batch) a.ws_prefix[b + 1] = carry + v;
+        carry += __shfl_sync(0xffffffffu, v, 31);
+        carry_v += __shfl_sync(0xffffffffu, vv, 31);
+    }
+    const long long total = (long long)carry * hkv, total_v = (long long)carry_v * hkv;
+    const long long xb = share_begin(blockIdx.x, total_v, gridDim.x);
+    const long long xe = share_begin(blockIdx.x + 1, total_v, gridDim.x);
+    // pass 2: cost positions -> tiles.  A position inside pair j of its sequence maps to that
+    // pair's tile at the same offset, or to the next pair's first tile if it falls in the cost part.
+    long long tb = total, te = total;
+    carry = carry_v = 0;
+    for (int base = 0; base < batch; base += 32) {
+        const int b = base + lane;
+        const int nt = (b < batch) ? seq_tiles(p, b, nullptr, false, tile) : 0;
+        const int w = nt > 0 ? nt + seg_cost : 0;
+        int v = nt, vv = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, v, d), tv = __shfl_up_sync(0xffffffffu, vv, d);
+            if (lane >= d) { v += t; vv += tv; }
+        }
+        const int pr = carry + v - nt, pv = carry_v + vv - w;
+        const long long lo = (long long)pv * hkv, hi = (long long)(pv + w) * hkv;
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+            const long long x = which == 0 ? xb : xe;
+            const unsigned hit = __ballot_sync(0xffffffffu, w > 0 && lo <= x && x < hi);
+            if (hit != 0) {
+                const int src = __ffs(hit) - 1;
+                const int s_nt = __shfl_sync(0xffffffffu, nt, src);
+                const int s_pr = __shfl_sync(0xffffffffu, pr, src), s_pv = __shfl_sync(0xffffffffu, pv, src);
+                const long long rem = x - (long long)s_pv * hkv;
+                const long long j = rem / (s_nt + seg_cost), off = rem - j * (s_nt + seg_cost);
+                const long long t = (long long)s_pr * hkv + j * s_nt + (off < s_nt ? off : s_nt);
+                if (which == 0) tb = t; else te = t;
+            }
+        }
+        carry += __shfl_sync(0xffffffffu, v, 31);
+        carry_v += __shfl_sync(0xffffffffu, vv, 31);
+    }
+    // pass 3: the sequence whose tiles contain the block's first tile
+    int sb = 0, sp = 0;
+    carry = 0;
+    for (int base = 0; base < batch; base += 32) {
+        const int b = base + lane;
+        const int nt = (b < batch) ? seq_tiles(p, b, nullptr, false, tile) : 0;
+        int v = nt;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, v, d);
+            if (lane >= d) v += t;
+        }
+        const long long lo = (long long)(carry + v - nt) * hkv, hi = (long long)(carry + v) * hkv;
+        const unsigned hit = __ballot_sync(0xffffffffu, nt > 0 && lo <= tb && tb < hi);
+        if (hit != 0) {
+            const int src = __ffs(hit) - 1;
+            sb = __shfl_sync(0xffffffffu, b, src);
+            sp = __shfl_sync(0xffffffffu, carry + v - nt, src);
+        }
+        carry += __shfl_sync(0xffffffffu, v, 31);
+    }
+    if (lane == 0) {
+        bounds[blockIdx.x] = (int)tb;
+        if (blockIdx.x + 1 == gridDim.x) bounds[gridDim.x] = (int)total;
+        if (blockIdx.x == 0) a.ws_prefix[batch + 1] = (int)gridDim.x;
+    }
+    o.total_tiles = carry;
+    o.t_begin = tb;
+    o.t_end = te;
+    o.start_b = sb;
+    o.start_prefix = sp;
 }
 
 // Walks the (sequence, kv head, tile) triples of a block's share.

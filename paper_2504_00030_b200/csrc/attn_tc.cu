@@ -50,6 +50,7 @@ struct Shared {
     int total_tiles;         // sum over sequences of ceil(L/128)
     int start_b;             // sequence that holds this block's first tile
     int start_prefix;        // tiles (per kv head) of the sequences before it
+    long long t_begin, t_end; // this block's tiles of the global list
 };
 
 
@@ -97,46 +98,14 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
     }
     __syncthreads();
     if (warp == 0) {
-        // pass 1: total tiles; block 0 also publishes the inclusive prefix for the combine kernel
-        int carry = 0;
-        if (blockIdx.x == 0 && lane == 0) a.ws_prefix[0] = 0;
-        for (int base = 0; base < batch; base += 32) {
-            const int b = base + lane;
-            int v = (b < batch) ? seq_tiles(p, b, nullptr, blockIdx.x == 0, TILE) : 0;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, v, d);
-                if (lane >= d) v += t;
-            }
-            if (blockIdx.x == 0 && b < batch) a.ws_prefix[b + 1] = carry + v;
-            carry += __shfl_sync(0xffffffffu, v, 31);
-        }
-        const long long total = (long long)carry * hkv;
-        const long long my_begin = share_begin(blockIdx.x, total, gridDim.x);
+        BlockShare bs;
+        plan_block_share(a, lane, TILE, 0, bs);
         if (lane == 0) {
-            sh->total_tiles = carry;
-            sh->start_b = 0;
-            sh->start_prefix = 0;
-            if (blockIdx.x == 0) a.ws_prefix[batch + 1] = (int)gridDim.x;
-        }
-        __syncwarp();
-        // pass 2: the sequence whose tiles contain this block's first tile
-        carry = 0;
-        for (int base = 0; base < batch; base += 32) {
-            const int b = base + lane;
-            const int nt = (b < batch) ? seq_tiles(p, b, nullptr, false, TILE) : 0;
-            int v = nt;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, v, d);
-                if (lane >= d) v += t;
-            }
-            const long long lo = (long long)(carry + v - nt) * hkv, hi = (long long)(carry + v) * hkv;
-            if (nt > 0 && lo <= my_begin && my_begin < hi) {
-                sh->start_b = b;
-                sh->start_prefix = carry + v - nt;
-            }
-            carry += __shfl_sync(0xffffffffu, v, 31);
+            sh->total_tiles = bs.total_tiles;
+            sh->t_begin = bs.t_begin;
+            sh->t_end = bs.t_end;
+            sh->start_b = bs.start_b;
+            sh->start_prefix = bs.start_prefix;
         }
     }
     if (warp == 1) {
@@ -152,8 +121,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
 
     const long long total = (long long)sh->total_tiles * hkv;
     const long long grid = gridDim.x;
-    const long long t_begin = share_begin(blockIdx.x, total, grid);
-    const long long t_end = share_begin(blockIdx.x + 1, total, grid);
+    const long long t_begin = sh->t_begin, t_end = sh->t_end;
     const uint32_t tmem = sh->tmem_base;
     const float c_scale = p.sm_scale * 1.4426950408889634f;   // scores in log2 units
 
@@ -530,12 +498,19 @@ attn_combine_kernel(const AttnTcLaunch a)
     const int n_tiles = a.ws_prefix[b + 1] - a.ws_prefix[b];
     if (n_tiles == 0 || total == 0) return;
     const long long T0 = (long long)a.ws_prefix[b] * p.hkv + (long long)g * n_tiles, T1 = T0 + n_tiles;
-    // blocks whose share contains tile T0 and tile T1-1
-    const long long c_first = ((T0 + 1) * grid + total - 1) / total - 1;
-    const long long c_last = (T1 * grid + total - 1) / total - 1;
-    if (c_first == c_last && share_begin(c_first, total, grid) <= T0 &&
-        share_begin(c_first + 1, total, grid) >= T1)
-        return;                                          // one block saw the whole pair: already final
+    // blocks whose share contains tile T0 and tile T1-1: the last block whose lower bound is not
+    // beyond the tile (empty shares repeat their successor's bound and are skipped that way)
+    const int32_t *bounds = a.ws_prefix + p.batch + 2;
+    auto owner = [&](long long t) {
+        long long lo = 0, hi = grid;
+        while (hi - lo > 1) {
+            const long long mid = (lo + hi) >> 1;
+            if (bounds[mid] <= t) lo = mid; else hi = mid;
+        }
+        return lo;
+    };
+    const long long c_first = owner(T0), c_last = owner(T1 - 1);
+    if (c_first == c_last) return;                       // one block saw the whole pair: already final
     int gam = p.gamma[b];
     gam = min(max(gam, 0), p.gamma_max);
     const int G = a.group, n_rows = G * (gam + 1);
@@ -554,8 +529,8 @@ attn_combine_kernel(const AttnTcLaunch a)
             if (carry >= 0) s_list[n++] = carry;
             long long c = c0;
             for (; c <= c_last && n < COMBINE_LIST; ++c) {
-                const long long lo = share_begin(c, total, grid);
-                if (share_begin(c + 1, total, grid) == lo) continue;
+                const long long lo = bounds[c];
+                if (bounds[c + 1] == lo) continue;
                 s_list[n++] = (int)(c * 2 + (lo >= T0 ? 0 : 1));
             }
             s_n = n;
@@ -632,7 +607,10 @@ bool attn_tc_supported(const sv_attn_params &p)
     return nq >= 1 && nq <= 2;
 }
 
-static size_t prefix_bytes(int batch) { return (((size_t)batch + 2) * sizeof(int32_t) + 255) & ~(size_t)255; }
+static size_t prefix_bytes(int batch)
+{
+    return (((size_t)batch + 2 + MAX_ATTN_GRID + 1) * sizeof(int32_t) + 255) & ~(size_t)255;
+}
 
 // blocks of the main kernel: two per SM with one row group (64-token tiles), else one per SM
 static int attn_grid(int nq) { return nq == 1 ? 2 * sm_count() : sm_count(); }
@@ -692,6 +670,7 @@ sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t worksp
     const bool use_tq = attn_tq_supported(p) && variant != 1;
     a.slot_rows = use_tq ? attn_tq_slot_rows(rows) : a.nq * 128;
     const int grid = use_tq ? sm_count() : attn_grid(a.nq);
+    if (grid > MAX_ATTN_GRID) return SV_EUNSUPPORTED;
     if (workspace_bytes < prefix_bytes(p.batch) + (size_t)grid * 2 * part_slot_floats(a.slot_rows) * sizeof(float))
         return SV_EWORKSPACE;
     a.ws_prefix = static_cast<int32_t *>(workspace);

@@ -37,6 +37,7 @@ constexpr int O_COL0 = 256;                        // the O accumulator,
 constexpr int Q_COL0 = 384;                        // the query rows (bf16 pairs)
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int TAIL_ROWS = 16;
+constexpr int SEG_COST = 4;                        // starting a pair costs about as much as four tiles (measured: 5.8 us against 1.5 us)
 constexpr float RESCALE_THRESHOLD = 8.f;           // log2 units: P <= 2^8 before a lazy rescale
 
 struct Shared {
@@ -50,6 +51,7 @@ struct Shared {
     uint32_t tmem_base;
     int abort_flag;
     int total_tiles;
+    long long t_begin, t_end;    // this block's tiles of the global list
     int start_b;
     int start_prefix;
 };
@@ -139,46 +141,14 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
     }
     __syncthreads();
     if (warp == 0) {
-        // pass 1: total tiles; block 0 also publishes the inclusive prefix for the combine kernel
-        int carry = 0;
-        if (blockIdx.x == 0 && lane == 0) a.ws_prefix[0] = 0;
-        for (int base = 0; base < batch; base += 32) {
-            const int b = base + lane;
-            int v = (b < batch) ? seq_tiles(p, b, nullptr, blockIdx.x == 0, TILE) : 0;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, v, d);
-                if (lane >= d) v += t;
-            }
-            if (blockIdx.x == 0 && b < batch) a.ws_prefix[b + 1] = carry + v;
-            carry += __shfl_sync(0xffffffffu, v, 31);
-        }
-        const long long total = (long long)carry * hkv;
-        const long long my_begin = share_begin(blockIdx.x, total, gridDim.x);
+        BlockShare bs;
+        plan_block_share(a, lane, TILE, SEG_COST, bs);
         if (lane == 0) {
-            sh->total_tiles = carry;
-            sh->start_b = 0;
-            sh->start_prefix = 0;
-            if (blockIdx.x == 0) a.ws_prefix[batch + 1] = (int)gridDim.x;
-        }
-        __syncwarp();
-        // pass 2: the sequence whose tiles contain this block's first tile
-        carry = 0;
-        for (int base = 0; base < batch; base += 32) {
-            const int b = base + lane;
-            const int nt = (b < batch) ? seq_tiles(p, b, nullptr, false, TILE) : 0;
-            int v = nt;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, v, d);
-                if (lane >= d) v += t;
-            }
-            const long long lo = (long long)(carry + v - nt) * hkv, hi = (long long)(carry + v) * hkv;
-            if (nt > 0 && lo <= my_begin && my_begin < hi) {
-                sh->start_b = b;
-                sh->start_prefix = carry + v - nt;
-            }
-            carry += __shfl_sync(0xffffffffu, v, 31);
+            sh->total_tiles = bs.total_tiles;
+            sh->t_begin = bs.t_begin;
+            sh->t_end = bs.t_end;
+            sh->start_b = bs.start_b;
+            sh->start_prefix = bs.start_prefix;
         }
     }
     if (warp == 1) {
@@ -194,8 +164,7 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
 
     const long long total = (long long)sh->total_tiles * hkv;
     const long long grid = gridDim.x;
-    const long long t_begin = share_begin(blockIdx.x, total, grid);
-    const long long t_end = share_begin(blockIdx.x + 1, total, grid);
+    const long long t_begin = sh->t_begin, t_end = sh->t_end;
     const uint32_t tmem = sh->tmem_base;
     const float c_scale = p.sm_scale * 1.4426950408889634f;   // scores in log2 units
     const int start_b = sh->start_b, start_prefix = sh->start_prefix;
