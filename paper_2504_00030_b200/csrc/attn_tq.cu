@@ -37,7 +37,7 @@ constexpr int O_COL0 = 256;                        // the O accumulator,
 constexpr int Q_COL0 = 384;                        // the query rows (bf16 pairs)
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int TAIL_ROWS = 16;
-constexpr int SEG_COST = 4;                        // starting a pair costs about as much as four tiles (measured: 5.8 us against 1.5 us)
+constexpr int SEG_COST = 6;                        // starting a pair costs about as much as six tiles (fitted: 5.8 us per pair against 1.5 us per tile; 3, 4 and 8 measured slower)
 constexpr float RESCALE_THRESHOLD = 8.f;           // log2 units: P <= 2^8 before a lazy rescale
 
 struct Shared {
