@@ -499,17 +499,24 @@ attn_combine_kernel(const AttnTcLaunch a)
     if (n_tiles == 0 || total == 0) return;
     const long long T0 = (long long)a.ws_prefix[b] * p.hkv + (long long)g * n_tiles, T1 = T0 + n_tiles;
     // blocks whose share contains tile T0 and tile T1-1: the last block whose lower bound is not
-    // beyond the tile (empty shares repeat their successor's bound and are skipped that way)
-    const int32_t *bounds = a.ws_prefix + p.batch + 2;
-    auto owner = [&](long long t) {
-        long long lo = 0, hi = grid;
+    // beyond the tile (empty shares repeat their successor's bound and are skipped that way).
+    // The table is copied to shared memory in one round trip and searched there.
+    __shared__ int s_bounds[MAX_ATTN_GRID + 1];
+    __shared__ int s_owner[2];
+    for (int c = threadIdx.x; c <= grid; c += blockDim.x) s_bounds[c] = a.ws_prefix[p.batch + 2 + c];
+    __syncthreads();
+    if (threadIdx.x < 2) {
+        const long long t = threadIdx.x == 0 ? T0 : T1 - 1;
+        int lo = 0, hi = (int)grid;
         while (hi - lo > 1) {
-            const long long mid = (lo + hi) >> 1;
-            if (bounds[mid] <= t) lo = mid; else hi = mid;
+            const int mid = (lo + hi) >> 1;
+            if (s_bounds[mid] <= t) lo = mid; else hi = mid;
         }
-        return lo;
-    };
-    const long long c_first = owner(T0), c_last = owner(T1 - 1);
+        s_owner[threadIdx.x] = lo;
+    }
+    __syncthreads();
+    const int *bounds = s_bounds;
+    const long long c_first = s_owner[0], c_last = s_owner[1];
     if (c_first == c_last) return;                       // one block saw the whole pair: already final
     int gam = p.gamma[b];
     gam = min(max(gam, 0), p.gamma_max);
