@@ -478,9 +478,9 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
 }
 
 // ---------------------------------------------------------------------------- combine kernel
-// One block per (sequence, kv head); merges the partials of pairs whose tiles were shared
-// by several blocks of the main kernel.  Warp = query row; a row's partials (running max, sum,
-// fp32 O) are all requested before the first is used, so a row costs one memory round trip.
+// Merges the partials of pairs whose tiles were shared by several blocks of the main kernel.
+// Warp = query row; a row's partials (running max, sum, fp32 O) are all requested before the
+// first is used, so a row costs one memory round trip.
 constexpr int COMBINE_THREADS = 1024;
 constexpr int COMBINE_LIST = 64;      // partial slots merged per pass
 
@@ -491,33 +491,46 @@ attn_combine_kernel(const AttnTcLaunch a)
     __shared__ int s_list[COMBINE_LIST];
     __shared__ int s_n;
     __shared__ long long s_next;
-    const int b = blockIdx.x / p.hkv, g = blockIdx.x % p.hkv;
+    // One block per block of the main kernel: block c looks at the tile where main block c's
+    // share began.  If that tile lies strictly inside a (sequence, kv head) pair, the pair was
+    // split there; the block whose bound is the FIRST one inside the pair merges it.
+    const int c = blockIdx.x;
     const int slot_rows = a.slot_rows;
     const long long grid = a.ws_prefix[p.batch + 1];
     const long long total = (long long)a.ws_prefix[p.batch] * p.hkv;
-    const int n_tiles = a.ws_prefix[b + 1] - a.ws_prefix[b];
-    if (n_tiles == 0 || total == 0) return;
-    const long long T0 = (long long)a.ws_prefix[b] * p.hkv + (long long)g * n_tiles, T1 = T0 + n_tiles;
-    // blocks whose share contains tile T0 and tile T1-1: the last block whose lower bound is not
-    // beyond the tile (empty shares repeat their successor's bound and are skipped that way).
-    // The table is copied to shared memory in one round trip and searched there.
+    if (c == 0 || c >= grid || total == 0) return;
+    // the table of lower bounds is copied to shared memory in one round trip and searched there
     __shared__ int s_bounds[MAX_ATTN_GRID + 1];
-    __shared__ int s_owner[2];
-    for (int c = threadIdx.x; c <= grid; c += blockDim.x) s_bounds[c] = a.ws_prefix[p.batch + 2 + c];
+    __shared__ int s_b, s_last;
+    for (int k = threadIdx.x; k <= grid; k += blockDim.x) s_bounds[k] = a.ws_prefix[p.batch + 2 + k];
+    if (threadIdx.x == 0) s_b = -1;
     __syncthreads();
-    if (threadIdx.x < 2) {
-        const long long t = threadIdx.x == 0 ? T0 : T1 - 1;
-        int lo = 0, hi = (int)grid;
+    const long long t = s_bounds[c];
+    if (t >= total) return;
+    for (int k = threadIdx.x; k < p.batch; k += blockDim.x) {      // the sequence that holds tile t
+        const long long lo = (long long)a.ws_prefix[k] * p.hkv, hi = (long long)a.ws_prefix[k + 1] * p.hkv;
+        if (lo <= t && t < hi) s_b = k;
+    }
+    __syncthreads();
+    const int b = s_b;
+    if (b < 0) return;
+    const int n_tiles = a.ws_prefix[b + 1] - a.ws_prefix[b];
+    const int g = (int)((t - (long long)a.ws_prefix[b] * p.hkv) / n_tiles);
+    const long long T0 = (long long)a.ws_prefix[b] * p.hkv + (long long)g * n_tiles, T1 = T0 + n_tiles;
+    if (t == T0 || s_bounds[c - 1] > T0) return;          // not split here, or an earlier bound is inside too
+    // shares that hold the pair's first and last tile: c - 1 (the last whose bound is not beyond
+    // T0; empty shares repeat their successor's bound and are skipped that way) and the owner of T1 - 1
+    if (threadIdx.x == 0) {
+        int lo = c, hi = (int)grid;
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
-            if (s_bounds[mid] <= t) lo = mid; else hi = mid;
+            if (s_bounds[mid] <= T1 - 1) lo = mid; else hi = mid;
         }
-        s_owner[threadIdx.x] = lo;
+        s_last = lo;
     }
     __syncthreads();
     const int *bounds = s_bounds;
-    const long long c_first = s_owner[0], c_last = s_owner[1];
-    if (c_first == c_last) return;                       // one block saw the whole pair: already final
+    const long long c_first = c - 1, c_last = s_last;
     int gam = p.gamma[b];
     gam = min(max(gam, 0), p.gamma_max);
     const int G = a.group, n_rows = G * (gam + 1);
@@ -686,7 +699,7 @@ sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t worksp
     if (use_tq) st = launch_attn_tq_main(a, p, grid, stream);
     else st = a.nq == 1 ? launch_main<1, 64>(a, p, grid, stream) : launch_main<2, 128>(a, p, grid, stream);
     if (st != SV_OK) return st;
-    attn_combine_kernel<<<p.batch * p.hkv, COMBINE_THREADS, 0, stream>>>(a);
+    attn_combine_kernel<<<grid, COMBINE_THREADS, 0, stream>>>(a);
     return launch_check();
 }
 
