@@ -65,6 +65,12 @@ def test_mixed_row_counts_around_128():
     check_attn(make_attn_case(cfg, gamma=np.full(20, 15, np.int32)))
 
 
+def test_more_than_144_rows_per_pair():
+    # 16 query heads per kv head x up to 13 positions = 208 rows: the kernel with two 128-row groups
+    cfg = synth.VerifyConfig("wide", 6, 32, 2, 128, 100, 200, 2600, 9, 12, 12, 1.0, 1.0, q_scale=3.0, seed=51)
+    check_attn(make_attn_case(cfg))
+
+
 def test_long_context_single_sequence():
     cfg = synth.VerifyConfig("long", 1, 8, 1, 128, 100, 16384, 16384, 16, 16, 16, 1.0, 1.0, q_scale=6.0,
                              seed=44)
