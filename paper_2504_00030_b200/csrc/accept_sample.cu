@@ -4,7 +4,7 @@
 //
 //  1. accept_rowstats_kernel -- the streaming pass and the only one that touches every
 //     logit.  Each (row, slice of the vocabulary) item is owned by ONE WARP: 128-bit
-//     streaming loads, eight per lane in flight, a single-pass online softmax with a
+//     streaming loads, six per lane in flight, a single-pass online softmax with a
 //     power-of-two running reference (so every rescale is exact), float32 ex2.approx
 //     exponentials summed four at a time into a float64 accumulator, and a warp-shuffle
 //     reduction at the end.  No block-level synchronisation at all.  Greedy sequences
@@ -29,7 +29,7 @@
 namespace sv {
 
 constexpr int RS_THREADS = 256;   // rowstats block (8 independent warps)
-constexpr int RS_UNROLL = 8;      // float4 loads in flight per lane
+constexpr int RS_UNROLL = 6;      // float4 loads in flight per lane: 61 registers, 32 warps per SM (4, 8, 12, 16 measured slower)
 constexpr int SEG = 128;          // vocabulary elements per sampling segment (one warp, float4 per lane)
 constexpr int SEG_THREADS = 256;
 constexpr int MAX_SPLITS = 16;    // blocks per sequence in the sampling kernel
