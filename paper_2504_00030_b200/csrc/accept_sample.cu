@@ -368,17 +368,27 @@ __device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideS
         if (greedy) {
             float v = first.amax;
             int ix = first.aidx;
-            for (int s = 1; s < a.n_slices; ++s) {
-                const RowPartial q = load_partial(pp + s);
-                merge_argmax(v, ix, q.amax, q.aidx);
+            for (int s0 = 1; s0 < a.n_slices; s0 += 4) {       // four records requested at once, merged in order
+                RowPartial q[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (s0 + u < a.n_slices) q[u] = load_partial(pp + s0 + u);
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (s0 + u < a.n_slices) merge_argmax(v, ix, q[u].amax, q[u].aidx);
             }
             sc->amax_idx[i] = ix;
         } else {
             float ref = first.ref;
             double sum = first.sum;
-            for (int s = 1; s < a.n_slices; ++s) {
-                const RowPartial q = load_partial(pp + s);
-                merge_stats(ref, sum, q.ref, q.sum);
+            for (int s0 = 1; s0 < a.n_slices; s0 += 4) {
+                RowPartial q[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (s0 + u < a.n_slices) q[u] = load_partial(pp + s0 + u);
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (s0 + u < a.n_slices) merge_stats(ref, sum, q[u].ref, q[u].sum);
             }
             sc->rref[j] = ref;
             sc->rsum[j] = sum;
