@@ -176,9 +176,10 @@ def gamma_tune_init(batch: int, gamma0: int, gamma_max: int = 0, padded_rows: bo
 
 
 def gamma_tune_update(n_accepted, gamma_bar, gamma, seq_len, eta, delta, gamma_min, gamma_max,
-                      mode=MODE_GT_PROPOSED, padded_rows=False):
+                      mode=MODE_GT_PROPOSED, padded_rows=False, n_drafted=None):
     """One controller update (Algorithm 1).  Returns NEW arrays
-    (gamma_bar, gamma, seq_len, cu_q, cu_d); the inputs are not modified."""
+    (gamma_bar, gamma, seq_len, cu_q, cu_d); the inputs are not modified.
+    n_drafted (GammaTune+): drafts actually produced this step, <= gamma."""
     lib = _load()
     A = _c(n_accepted, np.int32)
     B = len(A)
@@ -190,8 +191,29 @@ def gamma_tune_update(n_accepted, gamma_bar, gamma, seq_len, eta, delta, gamma_m
     lib.oracle_gamma_tune_update(_p(A), _p(gbar), _p(g), _p(sl), _p(cq), _p(cd), ctypes.c_int(B),
                                  ctypes.c_double(eta), ctypes.c_double(delta),
                                  ctypes.c_int(gamma_min), ctypes.c_int(gamma_max),
-                                 ctypes.c_int(mode), ctypes.c_int(int(padded_rows)))
+                                 ctypes.c_int(mode), ctypes.c_int(int(padded_rows)),
+                                 _p(_c(n_drafted, np.int32)) if n_drafted is not None else None)
     return gbar, g, sl, cq, cd
+
+
+DRAFT_STOP_TOL = 1e-6
+
+
+def draft_stop(draft_logits, temperature, tau, gamma, cu_d, tol=DRAFT_STOP_TOL):
+    """GammaTune+ early stop (Section 4.2): returns (n_drafted [B], top_prob [n_d_rows], flag [n_d_rows])."""
+    lib = _load()
+    dl = _c(draft_logits, np.float32)
+    g, cd = _c(gamma, np.int32), _c(cu_d, np.int32)
+    B = len(g)
+    T = np.broadcast_to(np.asarray(temperature, np.float32), (B,)).copy()
+    n_d = int(cd[B])
+    n = np.zeros(B, np.int32)
+    top = np.full(max(n_d, 1), np.nan)
+    flag = np.zeros(max(n_d, 1), np.uint8)
+    lib.oracle_draft_stop(_p(dl), ctypes.c_int64(dl.shape[1] if dl.ndim == 2 else 0), ctypes.c_int(dl.shape[1]),
+                          _p(T), ctypes.c_double(tau), _p(g), _p(cd), ctypes.c_int(B), ctypes.c_double(tol),
+                          _p(n), _p(top), _p(flag))
+    return n, top[:n_d], flag[:n_d]
 
 
 def cost_model(n_tokens, alpha, gamma, c):

@@ -1,6 +1,7 @@
 /*
  * Float64 CPU oracle for the speculative-decoding verify step
- * (attention of the draft block, accept / resample, GammaTune controller).
+ * (attention of the draft block, accept / resample, GammaTune controller,
+ * GammaTune+ early stop of drafting).
  *
  * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
  * CUDA library is checked against.  It shares no code with the CUDA path and
@@ -326,13 +327,17 @@ void oracle_accept_sample(const float *target_logits, const float *draft_logits,
 void oracle_gamma_tune_update(const int32_t *n_accepted, double *gamma_bar, int32_t *gamma,
                               int32_t *seq_len, int32_t *cu_q, int32_t *cu_d, int batch,
                               double eta, double delta, int gamma_min, int gamma_max, int mode,
-                              int padded_rows)
+                              int padded_rows, const int32_t *n_drafted)
 {
+    /* n_drafted (GammaTune+, Section 4.2; NULL for plain GammaTune): the draft stopped after
+     * n_drafted[b] <= gamma[b] tokens, so that many rows (+1) were appended to the cache; the
+     * comparison "A = gamma" still uses the gamma the controller issued. */
     cu_q[0] = 0;
     cu_d[0] = 0;
     for (int b = 0; b < batch; ++b) {
         int A = n_accepted[b];
         int g_old = gamma[b];
+        int rows_old = (n_drafted != NULL ? n_drafted[b] : g_old) + 1;
         int g_new = g_old;
         if (mode == 1 || mode == 2) {
             double a_eff = (double)A;
@@ -349,9 +354,45 @@ void oracle_gamma_tune_update(const int32_t *n_accepted, double *gamma_bar, int3
             g_new = (int)ceil(s);
         }
         gamma[b] = g_new;
-        seq_len[b] = seq_len[b] - (g_old + 1) + (A + 1) + (g_new + 1);
+        seq_len[b] = seq_len[b] - rows_old + (A + 1) + (g_new + 1);
         cu_q[b + 1] = padded_rows ? (b + 1) * (gamma_max + 1) : cu_q[b] + g_new + 1;
         cu_d[b + 1] = padded_rows ? (b + 1) * gamma_max : cu_d[b] + g_new;
+    }
+}
+
+/*
+ * GammaTune+ (Section 4.2): confidence-guided early stop of drafting.  The draft's confidence
+ * at position i is its top probability c_i = max_k softmax(d_i / T)_k.  The paper only says
+ * that drafting stops when it falls below tau; the reading taken here: the token drafted at
+ * the first such position is still part of the block, nothing is drafted after it, so
+ *     n_drafted = min(gamma, 1 + first i with c_i < tau)      (gamma if there is none).
+ * T = 0 (greedy draft): c_i = 1, never below tau <= 1.
+ * flag[row] = 1 when |c_i - tau| < tol (either decision is legal there).
+ */
+void oracle_draft_stop(const float *draft_logits, int64_t row_stride, int vocab, const float *temperature,
+                       double tau, const int32_t *gamma, const int32_t *cu_d, int batch, double tol,
+                       int32_t *n_drafted, double *top_prob, uint8_t *flag)
+{
+    for (int b = 0; b < batch; ++b) {
+        const int g = gamma[b];
+        const double T = (double)temperature[b];
+        int n = g;
+        for (int i = 0; i < g; ++i) {
+            const float *d = draft_logits + (int64_t)(cu_d[b] + i) * row_stride;
+            double c = 1.0;
+            if (T > 0.0) {
+                double m = -INFINITY;
+                for (int k = 0; k < vocab; ++k)
+                    if ((double)d[k] > m) m = (double)d[k];
+                double z = 0.0;
+                for (int k = 0; k < vocab; ++k) z += exp(((double)d[k] - m) / T);
+                c = 1.0 / z;
+            }
+            top_prob[cu_d[b] + i] = c;
+            flag[cu_d[b] + i] = fabs(c - tau) < tol ? 1 : 0;
+            if (n == g && c < tau) n = i + 1 < g ? i + 1 : g;
+        }
+        n_drafted[b] = n;
     }
 }
 
