@@ -13,6 +13,7 @@
  *                       token                                   (Section 3)
  *   gamma_tune_update   choose the next gamma from the number accepted
  *                                                               (Section 4.1, Algorithm 1)
+ * and, for GammaTune+, spec_draft_stop in front of them         (Section 4.2).
  *
  * General conventions
  *   - Pointers named "device" point to device memory owned by the caller; the
@@ -241,12 +242,52 @@ typedef struct sv_gamma_params {
     int32_t *accepted_log;      /* device out or NULL: A written to accepted_log[step*batch + b] */
     int32_t step;
     uint32_t *device_status;    /* device, one word or NULL */
+    const int32_t *n_drafted;   /* device [batch] or NULL: drafts actually produced this step when
+                                   drafting stopped early (spec_draft_stop); gamma[b] stays the
+                                   length the controller issued and is what A is compared with,
+                                   n_drafted[b]+1 is the number of positions the cache gained */
 } sv_gamma_params;
 
 sv_status gamma_tune_update(const sv_gamma_params *p, void *stream);
 /* gamma = gamma0 and gamma_bar = gamma0 for every sequence, cu_q / cu_d built; n_accepted,
  * seq_len, trajectory are not touched. */
 sv_status gamma_tune_init(const sv_gamma_params *p, int32_t gamma0, void *stream);
+
+/* ---------------------------------------------------------------- GammaTune+ early stop */
+/*
+ * Paper Section 4.2 (GammaTune+): drafting stops when the draft model's top
+ * probability falls below a threshold tau.  For sequence b and draft position
+ * i < gamma[b] the confidence is c_i = max_k softmax(d_i / T)_k (one streaming
+ * pass over the draft row: running max and sum).  The paper does not say
+ * whether the low-confidence token itself is kept; here it is, and nothing is
+ * drafted after it:
+ *     n_drafted[b] = min(gamma[b], 1 + first i with c_i < tau)   (gamma[b] if none).
+ * T == 0 (greedy draft): c_i = 1, drafting never stops early.
+ * The verify step then runs with n_drafted as its gamma array (attention,
+ * accept) and gamma_tune_update takes both (see sv_gamma_params.n_drafted).
+ * Confidences are float32 exponentials summed in float64; c_i and the
+ * comparison with tau are evaluated in float64.
+ */
+typedef struct sv_draft_stop_params {
+    const float *draft_logits;    /* device fp32 [n_d_rows, row_stride] */
+    int64_t row_stride;           /* elements between rows (>= vocab) */
+    int32_t vocab;
+    float temperature;            /* used when temperature_per_seq is NULL */
+    const float *temperature_per_seq; /* device [batch] or NULL */
+    float tau;                    /* threshold in [0, 1] */
+    const int32_t *gamma;         /* device [batch]: draft lengths issued by the controller */
+    const int32_t *cu_d;          /* device [batch+1] */
+    int32_t batch;
+    int32_t gamma_max;
+    int32_t *n_drafted;           /* device out [batch] */
+    double *top_prob;             /* device out [n_d_rows] or NULL: c_i of every draft row */
+    uint32_t *device_status;      /* device, one word or NULL */
+} sv_draft_stop_params;
+
+size_t spec_draft_stop_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t vocab);
+
+sv_status spec_draft_stop(const sv_draft_stop_params *p, void *workspace_device, size_t workspace_bytes,
+                          void *stream);
 
 /* ---------------------------------------------------------------- whole step from host buffers */
 /*

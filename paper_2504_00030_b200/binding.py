@@ -25,7 +25,7 @@ EXPORTS = (
     "sv_status_str", "sv_launch_count", "spec_kv_pool_register", "spec_kv_pool_release",
     "spec_verify_attn_workspace_bytes", "spec_verify_attn", "spec_accept_sample_workspace_bytes",
     "spec_accept_sample", "spec_accept_sample_static", "gamma_tune_update", "gamma_tune_init",
-    "spec_verify_step_host",
+    "spec_verify_step_host", "spec_draft_stop_workspace_bytes", "spec_draft_stop",
 )
 
 
@@ -64,7 +64,15 @@ class GammaParams(C.Structure):
     _fields_ = [("n_accepted", C.c_void_p), ("gamma_bar", C.c_void_p), ("gamma", C.c_void_p),
                 ("seq_len", C.c_void_p), ("cu_q", C.c_void_p), ("cu_d", C.c_void_p),
                 ("batch", C.c_int32), ("config", GammaConfigC), ("trajectory", C.c_void_p),
-                ("accepted_log", C.c_void_p), ("step", C.c_int32), ("device_status", C.c_void_p)]
+                ("accepted_log", C.c_void_p), ("step", C.c_int32), ("device_status", C.c_void_p),
+                ("n_drafted", C.c_void_p)]
+
+
+class DraftStopParams(C.Structure):
+    _fields_ = [("draft_logits", C.c_void_p), ("row_stride", C.c_int64), ("vocab", C.c_int32),
+                ("temperature", C.c_float), ("temperature_per_seq", C.c_void_p), ("tau", C.c_float),
+                ("gamma", C.c_void_p), ("cu_d", C.c_void_p), ("batch", C.c_int32), ("gamma_max", C.c_int32),
+                ("n_drafted", C.c_void_p), ("top_prob", C.c_void_p), ("device_status", C.c_void_p)]
 
 
 class StepHostIO(C.Structure):
@@ -110,6 +118,10 @@ def load():
         lib.gamma_tune_update.argtypes = [C.POINTER(GammaParams), C.c_void_p]
         lib.gamma_tune_init.restype = C.c_int32
         lib.gamma_tune_init.argtypes = [C.POINTER(GammaParams), C.c_int32, C.c_void_p]
+        lib.spec_draft_stop_workspace_bytes.restype = C.c_size_t
+        lib.spec_draft_stop_workspace_bytes.argtypes = [C.c_int32] * 3
+        lib.spec_draft_stop.restype = C.c_int32
+        lib.spec_draft_stop.argtypes = [C.POINTER(DraftStopParams), C.c_void_p, C.c_size_t, C.c_void_p]
         lib.spec_verify_step_host.restype = C.c_int32
         lib.spec_verify_step_host.argtypes = [C.POINTER(StepHostIO), C.POINTER(AttnParams), C.c_void_p,
                                               C.c_size_t, C.POINTER(AcceptParams), C.c_void_p,
@@ -318,7 +330,7 @@ class GammaConfig:
 
 
 def gamma_params(n_accepted, gamma_bar, gamma, seq_len, cu_q, cu_d, config: GammaConfig,
-                 trajectory=None, accepted_log=None, step=0, device_status=None) -> GammaParams:
+                 trajectory=None, accepted_log=None, step=0, device_status=None, n_drafted=None) -> GammaParams:
     p = GammaParams()
     p.n_accepted = _dev(n_accepted, torch.int32, "n_accepted", True)
     p.gamma_bar = _dev(gamma_bar, torch.float64, "gamma_bar")
@@ -333,15 +345,50 @@ def gamma_params(n_accepted, gamma_bar, gamma, seq_len, cu_q, cu_d, config: Gamm
     p.accepted_log = _dev(accepted_log, torch.int32, "accepted_log", True)
     p.step = step
     p.device_status = _dev(device_status, torch.int32, "device_status", True)
+    p.n_drafted = _dev(n_drafted, torch.int32, "n_drafted", True)
     return p
 
 
 def gamma_tune_update(n_accepted, gamma_bar, gamma, seq_len, cu_q, cu_d, config: GammaConfig,
-                      trajectory=None, accepted_log=None, step=0, device_status=None, stream=None):
+                      trajectory=None, accepted_log=None, step=0, device_status=None, stream=None,
+                      n_drafted=None):
     """One GammaTune update of every sequence's (gamma_bar, gamma) on the device (asynchronous)."""
     p = gamma_params(n_accepted, gamma_bar, gamma, seq_len, cu_q, cu_d, config, trajectory,
-                     accepted_log, step, device_status)
+                     accepted_log, step, device_status, n_drafted)
     _check("gamma_tune_update", load().gamma_tune_update(C.byref(p), _stream(stream)))
+
+
+# --------------------------------------------------------------------------- GammaTune+ early stop
+def spec_draft_stop_workspace_bytes(batch, gamma_max, vocab) -> int:
+    return int(load().spec_draft_stop_workspace_bytes(batch, gamma_max, vocab))
+
+
+def draft_stop_params(draft_logits, temperature, tau, gamma, cu_d, gamma_max, n_drafted, top_prob=None,
+                      device_status=None, temperature_per_seq=None) -> DraftStopParams:
+    p = DraftStopParams()
+    p.draft_logits = _dev(draft_logits, torch.float32, "draft_logits")
+    p.row_stride = draft_logits.stride(0)
+    p.vocab = draft_logits.shape[-1]
+    p.temperature = float(temperature)
+    p.temperature_per_seq = _dev(temperature_per_seq, torch.float32, "temperature_per_seq", True)
+    p.tau = float(tau)
+    p.gamma = _dev(gamma, torch.int32, "gamma")
+    p.cu_d = _dev(cu_d, torch.int32, "cu_d")
+    p.batch = gamma.shape[0]
+    p.gamma_max = gamma_max
+    p.n_drafted = _dev(n_drafted, torch.int32, "n_drafted")
+    p.top_prob = _dev(top_prob, torch.float64, "top_prob", True)
+    p.device_status = _dev(device_status, torch.int32, "device_status", True)
+    return p
+
+
+def spec_draft_stop(draft_logits, temperature, tau, gamma, cu_d, gamma_max, n_drafted, workspace,
+                    top_prob=None, device_status=None, temperature_per_seq=None, stream=None):
+    """GammaTune+ early stop of drafting: n_drafted per sequence (asynchronous)."""
+    p = draft_stop_params(draft_logits, temperature, tau, gamma, cu_d, gamma_max, n_drafted, top_prob,
+                          device_status, temperature_per_seq)
+    _check("spec_draft_stop",
+           load().spec_draft_stop(C.byref(p), workspace.data_ptr(), _nbytes(workspace), _stream(stream)))
 
 
 def gamma_tune_init(gamma_bar, gamma, cu_q, cu_d, config: GammaConfig, gamma0: int, stream=None):

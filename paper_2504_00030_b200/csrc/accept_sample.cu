@@ -36,7 +36,6 @@ constexpr int MAX_SPLITS = 16;    // blocks per sequence in the sampling kernel
 constexpr int MIN_SLICE = 2048;
 constexpr int MAX_SLICE = 16384;
 constexpr int MAX_GAMMA = 64;
-constexpr float REF_INIT = -1.0e30f;
 
 struct __align__(16) RowPartial {
     double sum;     // sum of 2^(x*c - ref) over the slice
@@ -91,22 +90,6 @@ __device__ __forceinline__ int seq_gamma(const sv_accept_params &p, int b)
         g = min(max(g, 0), p.gamma_max);
     }
     return g;
-}
-
-// x * 2^k for k <= 0, exact (x >= 0, normal or zero); far below the reference -> 0
-__device__ __forceinline__ double scale_down_pow2(double x, float k)
-{
-    if (!(k > -800.f) || !(x > 0.0)) return (x != x) ? x : 0.0;     // NaN stays NaN
-    if (k == 0.f || x == CUDART_INF) return x;
-    return __hiloint2double(__double2hiint(x) + ((int)k << 20), __double2loint(x));
-}
-
-// (ref, sum) pairs combine by rescaling to the larger reference; the factor is a power of two.
-__device__ __forceinline__ void merge_stats(float &ref, double &sum, float ref2, double sum2)
-{
-    const float r = fmaxf(ref, ref2);
-    sum = scale_down_pow2(sum, ref - r) + scale_down_pow2(sum2, ref2 - r);
-    ref = r;
 }
 
 __device__ __forceinline__ void merge_argmax(float &v, int &i, float v2, int i2)

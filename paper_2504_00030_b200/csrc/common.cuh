@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <math_constants.h>
 #include <stdint.h>
 
 #include "../../include/specverify.h"
@@ -74,6 +75,25 @@ __device__ __forceinline__ double warp_sum_f64(double v)
 #pragma unroll
     for (int m = 16; m > 0; m >>= 1) v += shfl_xor_f64(v, m);
     return v;
+}
+
+// ---- online softmax statistics shared by the kernels that stream logit rows
+constexpr float REF_INIT = -1.0e30f;    // running reference before the first element
+
+// x * 2^k for k <= 0, exact (x >= 0, normal or zero); far below the reference -> 0
+__device__ __forceinline__ double scale_down_pow2(double x, float k)
+{
+    if (!(k > -800.f) || !(x > 0.0)) return (x != x) ? x : 0.0;     // NaN stays NaN
+    if (k == 0.f || x == CUDART_INF) return x;
+    return __hiloint2double(__double2hiint(x) + ((int)k << 20), __double2loint(x));
+}
+
+// (ref, sum) pairs combine by rescaling to the larger reference; the factor is a power of two.
+__device__ __forceinline__ void merge_stats(float &ref, double &sum, float ref2, double sum2)
+{
+    const float r = fmaxf(ref, ref2);
+    sum = scale_down_pow2(sum, ref - r) + scale_down_pow2(sum2, ref2 - r);
+    ref = r;
 }
 
 }  // namespace sv

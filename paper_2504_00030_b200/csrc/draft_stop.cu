@@ -1,0 +1,238 @@
+// GammaTune+ confidence-guided early stop of drafting (paper Section 4.2).
+//
+// Two kernels on the caller's stream:
+//
+//  1. draft_conf_rowstats_kernel -- streams every draft row once.  One warp per (row, slice of
+//     the vocabulary): 128-bit streaming loads, six per lane in flight, running maximum of the
+//     logits and a single-pass online softmax sum with a power-of-two reference (float32
+//     ex2.approx exponentials accumulated in float64), warp-shuffle reduction, one record per
+//     item in the caller's workspace.
+//  2. draft_stop_decide_kernel -- one warp per sequence: merges the records of each draft
+//     position, evaluates the confidence c_i = 2^(max * log2(e)/T - ref) / sum in float64 and
+//     takes the first position below tau.
+#include "common.cuh"
+
+namespace sv {
+
+constexpr int DS_THREADS = 256;   // 8 independent warps
+constexpr int DS_UNROLL = 6;      // float4 loads in flight per lane
+constexpr int DS_MIN_SLICE = 2048;
+constexpr int DS_MAX_SLICE = 16384;
+constexpr int DS_MAX_GAMMA = 64;
+
+struct __align__(16) ConfPartial {
+    double sum;     // sum of 2^(x*c - ref) over the slice
+    float ref;      // integer-valued reference exponent
+    float amax;     // largest logit of the slice
+};
+
+struct DraftStopLaunch {
+    sv_draft_stop_params p;
+    ConfPartial *partials;   // [batch * gamma_max * n_slices]
+    int slice;               // elements per slice (multiple of 1024)
+    int n_slices;
+    int vec_ok;              // 128-bit loads legal for every row
+};
+
+__device__ __forceinline__ float ds_temperature(const sv_draft_stop_params &p, int b)
+{
+    return p.temperature_per_seq != nullptr ? p.temperature_per_seq[b] : p.temperature;
+}
+
+__device__ __forceinline__ int ds_gamma(const sv_draft_stop_params &p, int b)
+{
+    int g = p.gamma[b];
+    if (g < 0 || g > p.gamma_max) {
+        set_status(p.device_status, SV_DEV_BAD_GAMMA);
+        g = min(max(g, 0), p.gamma_max);
+    }
+    return g;
+}
+
+__global__ void __launch_bounds__(DS_THREADS)
+draft_conf_rowstats_kernel(const __grid_constant__ DraftStopLaunch a)
+{
+    const sv_draft_stop_params &p = a.p;
+    const long long n_items = (long long)p.batch * p.gamma_max * a.n_slices;
+    const int lane = threadIdx.x & 31;
+    const long long warp0 = (long long)blockIdx.x * (DS_THREADS / 32) + (threadIdx.x >> 5);
+    const long long n_warps = (long long)gridDim.x * (DS_THREADS / 32);
+
+    for (long long item = warp0; item < n_items; item += n_warps) {
+        const int slice_id = (int)(item % a.n_slices);
+        const int dense_row = (int)(item / a.n_slices);
+        const int b = dense_row / p.gamma_max, i = dense_row % p.gamma_max;
+        const float T = ds_temperature(p, b);
+        if (i >= ds_gamma(p, b) || !(T > 0.f)) continue;       // no such position, or a greedy draft
+        const float *row = p.draft_logits + (long long)(p.cu_d[b] + i) * p.row_stride;
+        const int lo = slice_id * a.slice;
+        const int hi = min(p.vocab, lo + a.slice);
+
+        // c = log2(e)/T split into a float pair with a strictly positive low part, so that
+        // x = -inf gives -inf (never inf - inf) and NaN / +inf inputs surface in the sum.
+        const double c = 1.4426950408889634 / (double)T;
+        float c_hi = __double2float_rd(c);
+        float c_lo = (float)(c - (double)c_hi);
+        if (!(c_lo > 0.f)) {
+            c_hi = __int_as_float(__float_as_int(c_hi) - 1);
+            c_lo = (float)(c - (double)c_hi);
+        }
+        float ref = REF_INIT, amax = -CUDART_INF_F;
+        double sum = 0.0;
+        auto consume4 = [&](float x0, float x1, float x2, float x3) {
+            const float m4 = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
+            amax = fmaxf(amax, m4);
+            const float ymax = m4 * c_hi + 1.f;
+            if (ymax > ref) {   // rare: the running reference has to grow
+                const float nr = ceilf(ymax);
+                sum = scale_down_pow2(sum, ref - nr);
+                ref = nr;
+            }
+            const float e0 = ex2_approx(fmaf(x0, c_lo, fmaf(x0, c_hi, -ref)));
+            const float e1 = ex2_approx(fmaf(x1, c_lo, fmaf(x1, c_hi, -ref)));
+            const float e2 = ex2_approx(fmaf(x2, c_lo, fmaf(x2, c_hi, -ref)));
+            const float e3 = ex2_approx(fmaf(x3, c_lo, fmaf(x3, c_hi, -ref)));
+            sum += (double)((e0 + e1) + (e2 + e3));
+        };
+        if (a.vec_ok) {
+            const int n4 = (hi - lo) >> 2;
+            const float *base = row + lo;
+            for (int v0 = lane; v0 < n4; v0 += 32 * DS_UNROLL) {
+                float4 x[DS_UNROLL];
+#pragma unroll
+                for (int u = 0; u < DS_UNROLL; ++u) {
+                    const int v = v0 + u * 32;
+                    x[u] = (v < n4) ? ld_stream_f4(base + 4 * (long long)v)
+                                    : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
+                }
+#pragma unroll
+                for (int u = 0; u < DS_UNROLL; ++u)
+                    if (v0 + u * 32 < n4) consume4(x[u].x, x[u].y, x[u].z, x[u].w);
+            }
+            const int tail0 = lo + 4 * n4;       // vocab not a multiple of 4: at most 3 elements, last slice only
+            if (lane == 0 && tail0 < hi) {
+                float t[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) t[u] = (tail0 + u < hi) ? row[tail0 + u] : -CUDART_INF_F;
+                consume4(t[0], t[1], t[2], t[3]);
+            }
+        } else {
+            for (int k0 = lo + 4 * lane; k0 < hi; k0 += 4 * 32) {
+                float t[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) t[u] = (k0 + u < hi) ? __ldg(row + k0 + u) : -CUDART_INF_F;
+                consume4(t[0], t[1], t[2], t[3]);
+            }
+        }
+        float r = ref;
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) {
+            r = fmaxf(r, __shfl_xor_sync(0xffffffffu, r, m));
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, m));
+        }
+        sum = warp_sum_f64(scale_down_pow2(sum, ref - r));
+        if (lane == 0) {
+            ConfPartial out;
+            out.sum = sum;
+            out.ref = r;
+            out.amax = amax;
+            a.partials[(long long)dense_row * a.n_slices + slice_id] = out;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(32)
+draft_stop_decide_kernel(const __grid_constant__ DraftStopLaunch a)
+{
+    const sv_draft_stop_params &p = a.p;
+    const int b = blockIdx.x, lane = threadIdx.x;
+    const int g = ds_gamma(p, b);
+    const float Tf = ds_temperature(p, b);
+    const double tau = (double)p.tau;
+    int first = g;                                     // first position whose confidence is below tau
+    for (int i0 = 0; i0 < g; i0 += 32) {
+        const int i = i0 + lane;
+        bool below = false;
+        if (i < g) {
+            double conf = 1.0;                         // greedy draft: the drafted token has probability one
+            if (Tf > 0.f) {
+                const ConfPartial *pp = a.partials + ((long long)b * p.gamma_max + i) * a.n_slices;
+                float ref = pp[0].ref, amax = pp[0].amax;
+                double sum = pp[0].sum;
+                for (int s = 1; s < a.n_slices; ++s) {
+                    merge_stats(ref, sum, pp[s].ref, pp[s].sum);
+                    amax = fmaxf(amax, pp[s].amax);
+                }
+                // top probability = exp(max/T) / sum_k exp(x_k/T) = 2^(max c - ref) / sum
+                conf = exp2((double)amax * (1.4426950408889634 / (double)Tf) - (double)ref) / sum;
+                if (!(conf == conf)) set_status(p.device_status, SV_DEV_NONFINITE);
+            }
+            if (p.top_prob != nullptr) p.top_prob[p.cu_d[b] + i] = conf;
+            below = conf < tau;
+        }
+        const unsigned m = __ballot_sync(0xffffffffu, below);
+        if (m != 0 && first == g) first = i0 + __ffs(m) - 1;
+    }
+    if (lane == 0) p.n_drafted[b] = first < g ? first + 1 : g;
+}
+
+static size_t ds_align256(size_t n) { return (n + 255) & ~(size_t)255; }
+
+static int ds_pick_slice(const sv_draft_stop_params *p)
+{
+    const long long rows = (long long)p->batch * p->gamma_max;
+    const long long want = 4LL * sm_count() * 32;
+    int slice = DS_MAX_SLICE;
+    while (slice > DS_MIN_SLICE && rows * ((p->vocab + slice - 1) / slice) < want) slice >>= 1;
+    return slice;
+}
+
+}  // namespace sv
+
+extern "C" size_t spec_draft_stop_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t vocab)
+{
+    if (batch <= 0 || gamma_max < 0 || vocab <= 0) return 0;
+    const size_t n_slices = ((size_t)vocab + sv::DS_MIN_SLICE - 1) / sv::DS_MIN_SLICE;
+    const size_t n = sv::ds_align256((size_t)batch * (size_t)gamma_max * n_slices * sizeof(sv::ConfPartial));
+    return n > 256 ? n : 256;
+}
+
+extern "C" sv_status spec_draft_stop(const sv_draft_stop_params *p, void *workspace, size_t workspace_bytes,
+                                     void *stream)
+{
+    if (p == nullptr || p->batch <= 0 || p->vocab <= 0 || p->gamma_max < 0) return SV_EINVAL;
+    if (p->gamma_max > sv::DS_MAX_GAMMA) return SV_EUNSUPPORTED;
+    if (p->gamma == nullptr || p->cu_d == nullptr || p->n_drafted == nullptr) return SV_EINVAL;
+    if (p->gamma_max > 0 && p->draft_logits == nullptr) return SV_EINVAL;
+    if (p->row_stride < p->vocab) return SV_EINVAL;
+    if (!(p->temperature >= 0.f) || !(p->tau >= 0.f) || !(p->tau <= 1.f)) return SV_EINVAL;
+    if (workspace == nullptr ||
+        workspace_bytes < spec_draft_stop_workspace_bytes(p->batch, p->gamma_max, p->vocab))
+        return SV_EWORKSPACE;
+    if (!sv::aligned16(workspace)) return SV_EALIGN;
+    cudaStream_t s = (cudaStream_t)stream;
+    sv::DraftStopLaunch a;
+    a.p = *p;
+    a.partials = static_cast<sv::ConfPartial *>(workspace);
+    a.slice = sv::ds_pick_slice(p);
+    a.n_slices = (p->vocab + a.slice - 1) / a.slice;
+    a.vec_ok = (p->row_stride % 4 == 0) && sv::aligned16(p->draft_logits);
+    const long long n_items = (long long)p->batch * p->gamma_max * a.n_slices;
+    if (n_items > 0) {
+        static int blocks_per_sm = 0;       // resident blocks per SM, asked once
+        if (blocks_per_sm == 0) {
+            int n = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, sv::draft_conf_rowstats_kernel, sv::DS_THREADS,
+                                                              0) != cudaSuccess || n < 1)
+                n = 2;
+            blocks_per_sm = n;
+        }
+        const long long blocks_needed = (n_items + sv::DS_THREADS / 32 - 1) / (sv::DS_THREADS / 32);
+        const long long cap = (long long)blocks_per_sm * sv::sm_count();
+        sv::draft_conf_rowstats_kernel<<<(int)(blocks_needed < cap ? blocks_needed : cap), sv::DS_THREADS, 0, s>>>(a);
+        const sv_status st = sv::launch_check();
+        if (st != SV_OK) return st;
+    }
+    sv::draft_stop_decide_kernel<<<p->batch, 32, 0, s>>>(a);
+    return sv::launch_check();
+}

@@ -58,6 +58,19 @@ gamma_tune_kernel(sv_gamma_params p, int gamma0)
                 }
                 int A = p.n_accepted[b];
                 A = min(max(A, 0), g_old);
+                // GammaTune+ (Section 4.2): the draft may have stopped after n_drafted <= gamma
+                // tokens; that many positions (+1) entered the cache, while "A = gamma" below
+                // still refers to the gamma this controller issued.
+                int rows_old = g_old + 1;
+                if (p.n_drafted != nullptr) {
+                    int nd = p.n_drafted[b];
+                    if (nd < 0 || nd > g_old) {
+                        set_status(p.device_status, SV_DEV_BAD_GAMMA);
+                        nd = min(max(nd, 0), g_old);
+                    }
+                    rows_old = nd + 1;
+                    A = min(A, nd);
+                }
                 g_new = g_old;
                 if (c.mode == SV_GT_PROPOSED || c.mode == SV_GT_LITERAL) {
                     // Eq. 7: the expansion raises the count fed to the average (proposed
@@ -75,7 +88,7 @@ gamma_tune_kernel(sv_gamma_params p, int gamma0)
                 }
                 p.gamma[b] = g_new;
                 if (p.seq_len != nullptr)
-                    p.seq_len[b] = p.seq_len[b] - (g_old + 1) + (A + 1) + (g_new + 1);
+                    p.seq_len[b] = p.seq_len[b] - rows_old + (A + 1) + (g_new + 1);
                 if (p.trajectory != nullptr) p.trajectory[(size_t)p.step * p.batch + b] = g_new;
                 if (p.accepted_log != nullptr) p.accepted_log[(size_t)p.step * p.batch + b] = A;
             }
