@@ -331,6 +331,23 @@ def run_ours(args):
     e2e_tokens = int((n_h + 1).sum().item())
     assert e2e_tokens == tokens
 
+    # ---- GammaTune+ early stop (not part of the step above): one streaming pass over the draft rows
+    n_dr = torch.zeros(B, dtype=torch.int32, device=DEV)
+    ws_d = torch.empty(max(256, sv.spec_draft_stop_workspace_bytes(B, gmax, cfg.vocab)), dtype=torch.uint8,
+                       device=DEV)
+    dp = sv.draft_stop_params(dl, cfg.temperature, 0.5, g, cd, gmax, n_dr, device_status=status)
+    state.copy_(state0)
+    ds_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(10)]
+    for _ in range(3):
+        check(lib.spec_draft_stop(C.byref(dp), ws_d.data_ptr(), ws_d.numel(), sptr), "draft_stop")
+    for e_a, e_b in ds_ev:
+        e_a.record(stream)
+        check(lib.spec_draft_stop(C.byref(dp), ws_d.data_ptr(), ws_d.numel(), sptr), "draft_stop")
+        e_b.record(stream)
+    barrier()
+    t_ds = float(np.median([e_a.elapsed_time(e_b) for e_a, e_b in ds_ev]))
+    ds_bytes = int(gamma.sum()) * cfg.vocab * 4
+
     # ---- reduce over ranks: max time, sum of tokens
     (ms_total, e2e_ms), tokens_all = shard.reduce_timing([ms_total, e2e_ms], tokens, device=DEV)
     if rank != 0:
@@ -364,6 +381,9 @@ def run_ours(args):
         "e2e": {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches), "clocks": clocks,
+        "draft_stop": {"what": "GammaTune+ early stop over the same draft rows, outside the timed step",
+                       "us": 1e3 * t_ds, "bytes": ds_bytes, "gbs": ds_bytes / (t_ds * 1e-3) / 1e9,
+                       "frac_of_measured": ds_bytes / (t_ds * 1e-3) / 1e9 / peak},
     }
     if world == 1 and not args.no_cpu_baseline:
         import oracle
