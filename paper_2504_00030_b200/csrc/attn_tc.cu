@@ -3,9 +3,9 @@
 // Work unit.  A (sequence b, kv head g) pair owns G*(gamma_b+1) query rows (G = hq/hkv query
 // heads per kv head, stacked so that the group shares one pass over the keys) and a stream of
 // ceil(L_b/128) key tiles of 128 tokens = 8 pages.  The key tiles of the whole batch form one
-// global list; each of the grid's persistent thread blocks takes an equal contiguous share of
-// it (lengths live on the device, so the split is computed in the kernel), which balances ragged
-// contexts exactly.  A block's share is cut into segments, one per (b, g) it touches; a segment
+// global list; each of the grid's persistent thread blocks takes a contiguous share of it
+// (lengths live on the device, so the split is computed in the kernel, see attn_sched.cuh),
+// which balances ragged contexts.  A block's share is cut into segments, one per (b, g) it touches; a segment
 // that covers its pair completely writes the final output, otherwise it leaves an unnormalised
 // partial (fp32 O, running max, running sum) in the workspace for attn_combine_kernel.
 //
