@@ -200,7 +200,8 @@ def run_ours(args):
     cfg, seq_len, gamma, cu_q, cu_d = workload_inputs(base_cfg, rank, args.batch, args.gamma, args.gamma_max)
     B, gmax = cfg.batch, cfg.gamma_max
     n_q, n_d = int(cu_q[-1]), int(cu_d[-1])
-    kv = synth.make_kv(cfg, seq_len, reserve_tokens=2 * (gmax + 1))
+    reserve = (2 + args.evolve) * (gmax + 1)
+    kv = synth.make_kv(cfg, seq_len, reserve_tokens=reserve)
     q_np = synth.make_q(cfg, n_q)
     li = synth.make_logits(cfg, gamma, cu_q, cu_d)
 
@@ -216,7 +217,7 @@ def run_ours(args):
     k_pool, v_pool = up_bf16(kv.k_pool), up_bf16(kv.v_pool)
     pool = sv.spec_kv_pool_register(k_pool, v_pool)
     bt = up(kv.block_table)
-    max_len = int(seq_len.max()) + 2 * (gmax + 1)
+    max_len = int(seq_len.max()) + reserve
     # host (pinned) copies of the per-step inputs for the end-to-end leg
     q_h = torch.from_numpy(q_np.view(np.int16)).view(torch.bfloat16).pin_memory()
     tl_h, dl_h = pin(li.target_logits), pin(li.draft_logits)
@@ -275,6 +276,19 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.evolve > 0:
+        # --evolve N: the controller runs N steps on its own acceptance counts first (no reset), and
+        # the timed steps start from the state it reached: a GammaTune-driven mix of draft lengths
+        # instead of gamma_max everywhere (the logit rows of a slab beyond a sequence's gamma are unused).
+        state.copy_(state0)
+        for _ in range(args.evolve):
+            check(lib.spec_verify_attn(C.byref(ap), ws_a.data_ptr(), ws_a.numel(), sptr), "attn")
+            check(lib.spec_accept_sample(C.byref(sp), ws_s.data_ptr(), ws_s.numel(), sptr), "accept")
+            check(lib.gamma_tune_update(C.byref(gp), sptr), "gamma")
+        torch.cuda.synchronize()
+        state0 = state.clone()
+        gamma = g.cpu().numpy().copy()
+        seq_len = sl.cpu().numpy().copy()
     for _ in range(args.warmup):
         step()
     barrier()
@@ -411,6 +425,8 @@ def main():
     ap.add_argument("--gamma", type=int, default=None,
                     help="draft length of every sequence (default: the workload's own range)")
     ap.add_argument("--gamma-max", type=int, default=None, help="override the controller's upper bound")
+    ap.add_argument("--evolve", type=int, default=0,
+                    help="let the controller run this many steps before the timed ones (a GammaTune-driven gamma mix)")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the workload's batch (smaller cases for profiler captures)")
     args = ap.parse_args()
