@@ -111,6 +111,29 @@ def verify_attn(q_bits, k_pool_bits, v_pool_bits, kv_strides, block_table, seq_l
     return o, lse
 
 
+def kv_append(k_new_bits, v_new_bits, k_pool_bits, v_pool_bits, kv_strides, block_table, seq_len, gamma,
+              cu_q, page_size):
+    """Write the draft block's keys and values behind each sequence's context.
+
+    k_new_bits, v_new_bits uint16 [sum R, hkv, D]; the pools are flat or shaped uint16 arrays
+    addressed through kv_strides (elements: page, head, slot, dim).  Returns modified copies of
+    the two pools; the arguments are left alone.
+    """
+    lib = _load()
+    kn, vn = _c(k_new_bits, np.uint16), _c(v_new_bits, np.uint16)
+    n_rows, hkv, D = kn.shape
+    assert vn.shape == kn.shape
+    assert k_pool_bits.dtype == np.uint16 and v_pool_bits.dtype == np.uint16
+    kp, vp = np.array(k_pool_bits, order="C", copy=True), np.array(v_pool_bits, order="C", copy=True)
+    st = _c(kv_strides, np.int64)
+    bt = _c(block_table, np.int32)
+    sl, g, cq = _c(seq_len, np.int32), _c(gamma, np.int32), _c(cu_q, np.int32)
+    lib.oracle_kv_append(_p(kn), _p(vn), _p(kp), _p(vp), _p(st), _p(bt), ctypes.c_int64(bt.shape[1]),
+                         _p(sl), _p(g), _p(cq), ctypes.c_int(len(sl)), ctypes.c_int(hkv), ctypes.c_int(D),
+                         ctypes.c_int(page_size))
+    return kp, vp
+
+
 # --------------------------------------------------------------------------- accept / resample
 @dataclass
 class AcceptResult:

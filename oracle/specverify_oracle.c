@@ -1,7 +1,7 @@
 /*
  * Float64 CPU oracle for the speculative-decoding verify step
- * (attention of the draft block, accept / resample, GammaTune controller,
- * GammaTune+ early stop of drafting).
+ * (appending the draft block to the paged cache, attention of the draft block,
+ * accept / resample, GammaTune controller, GammaTune+ early stop of drafting).
  *
  * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
  * CUDA library is checked against.  It shares no code with the CUDA path and
@@ -110,6 +110,39 @@ void oracle_verify_attn(const uint16_t *q, const uint16_t *k_pool, const uint16_
                             block_table + (int64_t)b * block_table_stride, page_size, h / group,
                             head_dim, pos + 1, scale, o + (row * hq + h) * head_dim,
                             lse ? lse + row * hq + h : NULL);
+        }
+    }
+}
+
+/* -------------------------------------------------------------------------
+ * 1b. Appending the draft block to the cache (KV caching, paper Section 5,
+ *     experimental setup).  Before the verify attention runs, the keys and
+ *     values of the gamma[b]+1 new positions are written behind the context:
+ *     new row i of sequence b is token  pos = seq_len[b] - (gamma[b]+1) + i
+ *     (seq_len already counts the block), which lives in physical page
+ *     block_table[b][pos / page_size], slot pos % page_size.  A plain copy of
+ *     bf16 bit patterns; every other element of the pools is left alone.
+ *     k_new, v_new: [sum R, hkv, head_dim].
+ * ------------------------------------------------------------------------- */
+void oracle_kv_append(const uint16_t *k_new, const uint16_t *v_new, uint16_t *k_pool, uint16_t *v_pool,
+                      const int64_t *kv_strides, const int32_t *block_table, int64_t block_table_stride,
+                      const int32_t *seq_len, const int32_t *gamma, const int32_t *cu_q, int batch,
+                      int hkv, int head_dim, int page_size)
+{
+    for (int b = 0; b < batch; ++b) {
+        int R = gamma[b] + 1;
+        for (int i = 0; i < R; ++i) {
+            int pos = seq_len[b] - R + i;
+            int64_t page = block_table[(int64_t)b * block_table_stride + pos / page_size];
+            int64_t slot = pos % page_size;
+            for (int g = 0; g < hkv; ++g) {
+                int64_t dst = page * kv_strides[0] + (int64_t)g * kv_strides[1] + slot * kv_strides[2];
+                int64_t src = (((int64_t)cu_q[b] + i) * hkv + g) * head_dim;
+                for (int d = 0; d < head_dim; ++d) {
+                    k_pool[dst + (int64_t)d * kv_strides[3]] = k_new[src + d];
+                    v_pool[dst + (int64_t)d * kv_strides[3]] = v_new[src + d];
+                }
+            }
         }
     }
 }
