@@ -122,6 +122,42 @@ size_t spec_verify_attn_workspace_bytes(int32_t batch, int32_t gamma_max, int32_
 sv_status spec_verify_attn(const sv_attn_params *p, void *workspace_device, size_t workspace_bytes,
                            void *stream);
 
+/* ---------------------------------------------------------------- cache append */
+/*
+ * KV caching (paper Section 5, experimental setup): before the verify
+ * attention runs, the keys and values of the gamma[b]+1 new positions are
+ * written behind each sequence's context.  New row i of sequence b (row
+ * cu_q[b]+i of k_new / v_new) is token
+ *     pos = seq_len[b] - (gamma[b]+1) + i
+ * (seq_len already counts the block) and goes to physical page
+ * block_table[b][pos / 16], slot pos % 16 of every kv head.  A copy of bf16
+ * bit patterns; nothing else in the pools is touched.  Rolling rejected
+ * positions back needs no copy: gamma_tune_update shortens seq_len, and the
+ * next append overwrites them.
+ * The pool memory (registered through const pointers for the attention) is
+ * written by this call; the caller owns it and orders the call before the
+ * attention on the same stream.
+ * Device-detected: gamma[b] out of range -> SV_DEV_BAD_GAMMA, clamped;
+ * seq_len[b] < gamma[b]+1 or a position beyond the block table row ->
+ * SV_DEV_BAD_LEN, sequence skipped; a page id outside [0, n_pages) ->
+ * SV_DEV_BAD_PAGE, that position skipped.
+ */
+typedef struct sv_kv_append_params {
+    const void *k_new;          /* device bf16 [n_rows, hkv, head_dim], 16-byte aligned */
+    const void *v_new;          /* device bf16 [n_rows, hkv, head_dim], 16-byte aligned */
+    sv_kv_pool_t pool;          /* head_dim a multiple of 8 */
+    const int32_t *block_table; /* device [batch, block_table_stride] */
+    int64_t block_table_stride;
+    const int32_t *seq_len;     /* device [batch] */
+    const int32_t *gamma;       /* device [batch] */
+    const int32_t *cu_q;        /* device [batch+1] */
+    int32_t batch;
+    int32_t gamma_max;          /* upper bound of gamma[b]; sizes the grid */
+    uint32_t *device_status;    /* device, one word, OR-ed into; may be NULL */
+} sv_kv_append_params;
+
+sv_status spec_kv_append(const sv_kv_append_params *p, void *stream);
+
 /* ---------------------------------------------------------------- accept / resample */
 /*
  * Speculative sampling (paper Section 3, after Leviathan et al. and Chen et

@@ -25,7 +25,7 @@ EXPORTS = (
     "sv_status_str", "sv_launch_count", "spec_kv_pool_register", "spec_kv_pool_release",
     "spec_verify_attn_workspace_bytes", "spec_verify_attn", "spec_accept_sample_workspace_bytes",
     "spec_accept_sample", "spec_accept_sample_static", "gamma_tune_update", "gamma_tune_init",
-    "spec_verify_step_host", "spec_draft_stop_workspace_bytes", "spec_draft_stop",
+    "spec_verify_step_host", "spec_draft_stop_workspace_bytes", "spec_draft_stop", "spec_kv_append",
 )
 
 
@@ -42,6 +42,13 @@ class AttnParams(C.Structure):
                 ("batch", C.c_int32), ("gamma_max", C.c_int32), ("hq", C.c_int32),
                 ("hkv", C.c_int32), ("head_dim", C.c_int32), ("max_seq_len", C.c_int32),
                 ("sm_scale", C.c_float), ("device_status", C.c_void_p)]
+
+
+class KvAppendParams(C.Structure):
+    _fields_ = [("k_new", C.c_void_p), ("v_new", C.c_void_p), ("pool", C.c_void_p),
+                ("block_table", C.c_void_p), ("block_table_stride", C.c_int64),
+                ("seq_len", C.c_void_p), ("gamma", C.c_void_p), ("cu_q", C.c_void_p),
+                ("batch", C.c_int32), ("gamma_max", C.c_int32), ("device_status", C.c_void_p)]
 
 
 class AcceptParams(C.Structure):
@@ -253,6 +260,34 @@ def spec_verify_attn(q, o, pool, block_table, seq_len, gamma, cu_q, gamma_max, m
                     sm_scale, lse, device_status)
     _check("spec_verify_attn",
            load().spec_verify_attn(C.byref(p), workspace.data_ptr(), _nbytes(workspace), _stream(stream)))
+
+
+def kv_append_params(k_new, v_new, pool, block_table, seq_len, gamma, cu_q, gamma_max,
+                     device_status=None) -> KvAppendParams:
+    p = KvAppendParams()
+    p.k_new = _dev(k_new, torch.bfloat16, "k_new")
+    p.v_new = _dev(v_new, torch.bfloat16, "v_new")
+    if tuple(k_new.shape) != tuple(v_new.shape) or k_new.dim() != 3:
+        raise ValueError("k_new and v_new must both be [n_rows, hkv, head_dim]")
+    if tuple(k_new.shape[1:]) != (pool.hkv, pool.head_dim):
+        raise ValueError("k_new rows do not match the pool's heads and head_dim")
+    p.pool = pool.handle
+    p.block_table = _dev(block_table, torch.int32, "block_table")
+    p.block_table_stride = block_table.shape[1]
+    p.seq_len = _dev(seq_len, torch.int32, "seq_len")
+    p.gamma = _dev(gamma, torch.int32, "gamma")
+    p.cu_q = _dev(cu_q, torch.int32, "cu_q")
+    p.batch = gamma.shape[0]
+    p.gamma_max = gamma_max
+    p.device_status = _dev(device_status, torch.int32, "device_status", True)
+    return p
+
+
+def spec_kv_append(k_new, v_new, pool, block_table, seq_len, gamma, cu_q, gamma_max, device_status=None,
+                   stream=None):
+    """Write the draft block's keys and values behind each sequence's context (asynchronous)."""
+    p = kv_append_params(k_new, v_new, pool, block_table, seq_len, gamma, cu_q, gamma_max, device_status)
+    _check("spec_kv_append", load().spec_kv_append(C.byref(p), _stream(stream)))
 
 
 # --------------------------------------------------------------------------- accept / resample
