@@ -362,6 +362,62 @@ def run_ours(args):
     t_ds = float(np.median([e_a.elapsed_time(e_b) for e_a, e_b in ds_ev]))
     ds_bytes = int(gamma.sum()) * cfg.vocab * 4
 
+    # ---- cache append (not part of the step above): the block's keys and values written behind the contexts
+    n_kv = n_q * cfg.hkv * cfg.head_dim
+    k_new = up_bf16(synth.normal_bf16_bits(cfg.seed, 90, n_kv).reshape(n_q, cfg.hkv, cfg.head_dim))
+    v_new = up_bf16(synth.normal_bf16_bits(cfg.seed, 91, n_kv).reshape(n_q, cfg.hkv, cfg.head_dim))
+    kp = sv.kv_append_params(k_new, v_new, pool, bt, sl, g, cq, gmax, device_status=status)
+    state.copy_(state0)
+    ka_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(10)]
+    for _ in range(3):
+        check(lib.spec_kv_append(C.byref(kp), sptr), "kv_append")
+    for e_a, e_b in ka_ev:
+        e_a.record(stream)
+        check(lib.spec_kv_append(C.byref(kp), sptr), "kv_append")
+        e_b.record(stream)
+    barrier()
+    t_ka = float(np.median([e_a.elapsed_time(e_b) for e_a, e_b in ka_ev]))
+    ka_bytes = int((gamma + 1).sum()) * cfg.hkv * cfg.head_dim * 2 * 2 * 2      # K and V, read and written
+
+    # ---- --layers N: N caches of the same shape behind one block table; every step appends to and
+    # attends over each of them in turn, then accepts and updates once (a model's worth of layers)
+    layers = None
+    if args.layers > 1:
+        pools = [pool]
+        keep = []
+        for _ in range(args.layers - 1):
+            kk, vv = k_pool.clone(), v_pool.clone()
+            keep.append((kk, vv))
+            pools.append(sv.spec_kv_pool_register(kk, vv))
+        aps = [sv.attn_params(q, o, pl, bt, sl, g, cq, gmax, max_len, device_status=status) for pl in pools]
+        kps = [sv.kv_append_params(k_new, v_new, pl, bt, sl, g, cq, gmax, device_status=status) for pl in pools]
+
+        def layer_step(ev=None):
+            state.copy_(state0, non_blocking=True)
+            if ev is not None: ev[0].record(stream)
+            for a_l, k_l in zip(aps, kps):
+                check(lib.spec_kv_append(C.byref(k_l), sptr), "kv_append")
+                check(lib.spec_verify_attn(C.byref(a_l), ws_a.data_ptr(), ws_a.numel(), sptr), "attn")
+            if ev is not None: ev[1].record(stream)
+            check(lib.spec_accept_sample(C.byref(sp), ws_s.data_ptr(), ws_s.numel(), sptr), "accept")
+            check(lib.gamma_tune_update(C.byref(gp), sptr), "gamma")
+            if ev is not None: ev[2].record(stream)
+
+        n_ls = max(3, min(args.steps, 20))
+        for _ in range(3):
+            layer_step()
+        barrier()
+        l_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_ls)]
+        for it in range(n_ls):
+            layer_step(l_ev[it])
+        barrier()
+        assert status.item() == 0, f"device status {status.item()}"
+        t_layers = float(np.mean([e[0].elapsed_time(e[1]) for e in l_ev]))
+        t_lstep = float(np.mean([e[0].elapsed_time(e[2]) for e in l_ev]))
+        layers = {"n": args.layers, "steps": n_ls, "us_per_layer": 1e3 * t_layers / args.layers,
+                  "step_us": 1e3 * t_lstep,
+                  "gbs": args.layers * synth.algorithmic_bytes(cfg, seq_len, gamma)[0] / (t_layers * 1e-3) / 1e9}
+
     # ---- reduce over ranks: max time, sum of tokens
     (ms_total, e2e_ms), tokens_all = shard.reduce_timing([ms_total, e2e_ms], tokens, device=DEV)
     if rank != 0:
@@ -399,6 +455,11 @@ def run_ours(args):
                        "us": 1e3 * t_ds, "bytes": ds_bytes, "gbs": ds_bytes / (t_ds * 1e-3) / 1e9,
                        "frac_of_measured": ds_bytes / (t_ds * 1e-3) / 1e9 / peak},
     }
+    line["kv_append"] = {"what": "the block's keys and values written into the paged cache, outside the timed step",
+                         "us": 1e3 * t_ka, "bytes": ka_bytes}
+    if layers is not None:
+        layers["frac_of_measured"] = layers["gbs"] / peak
+        line["layers"] = layers
     if world == 1 and not args.no_cpu_baseline:
         import oracle
         n_seq = min(args.oracle_seqs or 16, B)
@@ -427,6 +488,8 @@ def main():
     ap.add_argument("--gamma-max", type=int, default=None, help="override the controller's upper bound")
     ap.add_argument("--evolve", type=int, default=0,
                     help="let the controller run this many steps before the timed ones (a GammaTune-driven gamma mix)")
+    ap.add_argument("--layers", type=int, default=1,
+                    help="also time steps that append to and attend over this many caches in turn (memory: one KV pool each)")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the workload's batch (smaller cases for profiler captures)")
     args = ap.parse_args()
