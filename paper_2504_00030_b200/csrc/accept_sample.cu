@@ -135,7 +135,9 @@ __device__ const double g_exp2_table[128] = {
 
 // 2^y in float64 for y <= ~4 (anything below -1000, -inf or NaN gives 0).  y is split into
 // k/128 + r with k = rint(128 y): 2^y = 2^(k >> 7) * table[k & 127] * 2^r, |r| <= 1/256, 2^r by
-// its degree-5 Taylor polynomial (truncation below 1e-18); the power of two goes straight
+// its degree-3 Taylor polynomial: the first dropped term is (r ln 2)^4 / 24 <= 2.2e-12, a relative
+// error far below the 1e-9 window inside which a sampled token counts as a near tie, and common
+// to numerator and denominator of every cumulative fraction.  The power of two goes straight
 // into the exponent field.  N values at once, each step taken for all of them before the
 // next, so that the N dependent chains overlap in the pipeline; no branches.  `tab` is a
 // shared-memory copy of g_exp2_table.
@@ -152,12 +154,11 @@ __device__ __forceinline__ void exp2_f64_n(const double (&y)[N], double (&out)[N
         k[i] = __double2loint(m);
         r[i] = fma(m - MAGIC, -0.0078125, yc);
         t[i] = tab[k[i] & 127];
-        q[i] = 0.0013333558146428441;
+        q[i] = 0.055504108664821576;                  // (ln 2)^3 / 6
     }
-    constexpr double C[5] = {0.009618129107628477, 0.055504108664821576, 0.2402265069591007,
-                             0.6931471805599453, 1.0};
+    constexpr double C[3] = {0.2402265069591007, 0.6931471805599453, 1.0};
 #pragma unroll
-    for (int c = 0; c < 5; ++c)
+    for (int c = 0; c < 3; ++c)
 #pragma unroll
         for (int i = 0; i < N; ++i) q[i] = fma(q[i], r[i], C[c]);
 #pragma unroll
@@ -640,7 +641,7 @@ accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
     const bool vec = a.vec_ok != 0;
     const double ref_p = (double)rec.ref_p, ref_q = (double)rec.ref_q;
     // first-pass partition sums, good to ~1e-7: only used to decide the sign of p_k - q_k
-    const double inv_zp_hat = 1.0 / rec.sum_p_hat, inv_zq_hat = 1.0 / rec.sum_q_hat;
+    const double z_ratio = rec.sum_q_hat / rec.sum_p_hat;     // p_k > q_k  <=>  a_k * Zq > b_k * Zp
     double *seg_ap = a.seg + (size_t)b * 3 * n_seg, *seg_bp = seg_ap + n_seg, *seg_a = seg_bp + n_seg;
 
     const int per = (n_seg + a.splits - 1) / a.splits;
@@ -677,7 +678,7 @@ accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
                     const double ak = w[u], bk = w[4 + u];
                     sa += ak;
                     sb += bk;
-                    if (ak * inv_zp_hat > bk * inv_zq_hat) { sap += ak; sbp += bk; }
+                    if (ak * z_ratio > bk) { sap += ak; sbp += bk; }
                 }
             } else {
                 double y[4], w[4];
@@ -689,9 +690,24 @@ accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
             }
             tot_a += sa;
             tot_b += sb;
-            sa = warp_sum_f64(sa);
-            if (residual) { sap = warp_sum_f64(sap); sbp = warp_sum_f64(sbp); }
-            if (lane == 0) { seg_a[s] = sa; seg_ap[s] = sap; seg_bp[s] = sbp; }
+            if (residual) {
+                // the three sums in one butterfly: after the first exchange the lower half-warp
+                // carries (sa, sap) and the upper half sbp; after the second each quarter carries
+                // one of them; the totals end in lanes 0, 8 and 16
+                const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0;
+                double x0 = (up16 ? sbp : sa) + shfl_xor_f64(up16 ? sa : sbp, 16);
+                double x1 = (up16 ? 0.0 : sap) + shfl_xor_f64(up16 ? sap : 0.0, 16);
+                double y1 = (up8 ? x1 : x0) + shfl_xor_f64(up8 ? x0 : x1, 8);
+                y1 += shfl_xor_f64(y1, 4);
+                y1 += shfl_xor_f64(y1, 2);
+                y1 += shfl_xor_f64(y1, 1);
+                if (lane == 0) seg_a[s] = y1;
+                if (lane == 8) seg_ap[s] = y1;
+                if (lane == 16) seg_bp[s] = y1;
+            } else {
+                sa = warp_sum_f64(sa);
+                if (lane == 0) { seg_a[s] = sa; seg_ap[s] = 0.0; seg_bp[s] = 0.0; }
+            }
         }
     }
     tot_a = warp_sum_f64(tot_a);
