@@ -12,10 +12,11 @@ from tests.harness import (ATTN_ATOL, DEV, AcceptOut, bits_of, compare_accept, d
 pytestmark = pytest.mark.gpu
 
 
-def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0):
+def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0, append=False):
     """Runs `steps` verify steps on the device with padded row slabs; every per-step input is
     uploaded before the loop and nothing is read back until it ends.  Returns what the
-    oracle needs to replay the same steps, and the device's logs."""
+    oracle needs to replay the same steps, and the device's logs.  With `append` every step
+    first writes that step's new keys and values behind the contexts (spec_kv_append)."""
     B, gmax = cfg.batch, cfg.gamma_max
     cu_q, cu_d = synth.padded_offsets(B, gmax)
     n_q, n_d = int(cu_q[-1]), int(cu_d[-1])
@@ -29,6 +30,11 @@ def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0):
     inputs = [synth.make_logits(cfg, full_gamma, cu_q, cu_d, step=t, sigma_noise=sigmas[t % len(sigmas)])
               for t in range(steps)]
     qs = [synth.make_q(cfg, n_q, step=t) for t in range(steps)]
+    n_kv = n_q * cfg.hkv * cfg.head_dim
+    kv_new = [(synth.normal_bf16_bits(cfg.seed, 90, n_kv, 1.0, t).reshape(n_q, cfg.hkv, cfg.head_dim),
+               synth.normal_bf16_bits(cfg.seed, 91, n_kv, 1.0, t).reshape(n_q, cfg.hkv, cfg.head_dim))
+              for t in range(steps)] if append else []
+    d_kv = [(dev_bf16(a), dev_bf16(b)) for a, b in kv_new]
     d_in = [(dev(li.target_logits), dev(li.draft_logits), dev(li.draft_tokens), dev(li.u_accept),
              dev(li.u_sample), dev_bf16(q)) for li, q in zip(inputs, qs)]
 
@@ -49,6 +55,8 @@ def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0):
     sl0 = sl.clone()
     for t in range(steps):
         tl, dl, x, ua, us, q = d_in[t]
+        if append:
+            sv.spec_kv_append(d_kv[t][0], d_kv[t][1], pool, bt, sl, g, d_cq, gmax, device_status=status)
         sv.spec_verify_attn(q, o[t], pool, bt, sl, g, d_cq, gmax, max_len, ws_a, device_status=status)
         sv.spec_accept_sample(tl, dl, x, ua, us, cfg.temperature, g, d_cq, d_cd, gmax, n_acc, toks[t], ws_s,
                               device_status=status)
@@ -58,7 +66,8 @@ def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0):
     assert status.item() == 0
     return dict(kv=kv, inputs=inputs, qs=qs, cu_q=cu_q, cu_d=cu_d, sl0=sl0.cpu().numpy(),
                 toks=toks.cpu().numpy(), n_log=n_log.cpu().numpy(), traj=traj.cpu().numpy(),
-                o=o, gbar=gbar.cpu().numpy(), sl=sl.cpu().numpy())
+                o=o, gbar=gbar.cpu().numpy(), sl=sl.cpu().numpy(), kv_new=kv_new,
+                k_pool=bits_of(k) if append else None, v_pool=bits_of(v) if append else None)
 
 
 def replay_with_oracle(cfg, run, steps, gamma0, gcfg, check_attn_steps=()):
@@ -67,13 +76,17 @@ def replay_with_oracle(cfg, run, steps, gamma0, gcfg, check_attn_steps=()):
     sl = run["sl0"].copy()
     flagged = 0
     scale = float(np.float32(cfg.head_dim ** -0.5))
+    kp, vp = run["kv"].k_pool, run["kv"].v_pool
     for t in range(steps):
         li = run["inputs"][t]
+        if run["kv_new"]:
+            kp, vp = oracle.kv_append(run["kv_new"][t][0], run["kv_new"][t][1], kp, vp, run["kv"].strides,
+                                      run["kv"].block_table, sl, g, run["cu_q"], cfg.page_size)
         gpu = AcceptOut(run["n_log"][t], run["toks"][t], None, None, None, 0, 0)
         ref, n_pos, n_tok = compare_accept(gpu, li, cfg.temperature, g, run["cu_q"], run["cu_d"], gmax)
         flagged += n_pos + n_tok
         if t in check_attn_steps:
-            o_ref, _ = oracle.verify_attn(run["qs"][t], run["kv"].k_pool, run["kv"].v_pool, run["kv"].strides,
+            o_ref, _ = oracle.verify_attn(run["qs"][t], kp, vp, run["kv"].strides,
                                           run["kv"].block_table, sl, g, run["cu_q"], cfg.hq, cfg.hkv,
                                           cfg.page_size, scale)
             o_gpu = synth.bf16_to_f32(bits_of(run["o"][t])).astype(np.float64)
@@ -86,6 +99,10 @@ def replay_with_oracle(cfg, run, steps, gamma0, gcfg, check_attn_steps=()):
         np.testing.assert_array_equal(run["traj"][t], g)
     np.testing.assert_array_equal(run["gbar"].view(np.int64), gbar.view(np.int64))
     np.testing.assert_array_equal(run["sl"], sl)
+    if run["kv_new"]:
+        # the caches after the last step: every append, and every overwrite of a rejected position
+        np.testing.assert_array_equal(run["k_pool"], kp)
+        np.testing.assert_array_equal(run["v_pool"], vp)
     return flagged
 
 
@@ -114,6 +131,19 @@ def test_c4_alternating_regimes_reduced(T):
     easy = run["traj"][4:8].mean()
     hard = run["traj"][12:16].mean()
     assert easy > hard                                  # expands when drafts are accepted, contracts otherwise
+
+
+def test_loop_that_appends_each_block_to_the_cache():
+    # Llama-8B-like GQA shape, reduced: every step writes its block's keys and values, the controller
+    # drops the rejected positions by shortening seq_len, and the next block lands on top of them
+    cfg = synth.scaled(synth.CONFIGS["c3"], batch=3, hq=8, hkv=2, ctx_lo=200, ctx_hi=200, vocab=4000)
+    gcfg = sv.GammaConfig(0.5, 2.0, 1, cfg.gamma_max, sv.SV_GT_PROPOSED, True)
+    steps = 20
+    sig = [0.3] * 5 + [2.5] * 5
+    run = run_loop(cfg, steps, 4, gcfg, sig, 200, append=True)
+    replay_with_oracle(cfg, run, steps, 4, gcfg, check_attn_steps=(0, 7, 19))
+    assert (run["n_log"] < run["traj"].max()).any()     # there were rejections to roll back
+    assert (run["k_pool"] != run["kv"].k_pool).any()
 
 
 def test_step_from_host_buffers_matches_device_calls():
