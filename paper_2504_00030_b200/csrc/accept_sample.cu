@@ -9,8 +9,8 @@
 //     exponentials summed four at a time into a float64 accumulator, and a warp-shuffle
 //     reduction at the end.  No block-level synchronisation at all.  Greedy sequences
 //     (T = 0) only track (max, lowest index) of their target rows.
-//  2. accept_decide_kernel -- one warp per sequence: merges the slice statistics into ln Z
-//     per row (float64), evaluates ratio_i = min(1, p_i[x_i]/q_i[x_i]) against u_i in float64
+//  2. accept_decide_kernel -- one block per sequence: its warps merge the slice statistics
+//     into ln Z per row (float64, lanes over slices), then one warp evaluates ratio_i = min(1, p_i[x_i]/q_i[x_i]) against u_i in float64
 //     for all positions in parallel, then takes the first rejection.
 //  3. accept_sample_kernel -- several blocks per sequence: float64 pass over the one or two
 //     rows the next token is drawn from (residual max(0, p_n - q_n) or the bonus row), sums
@@ -32,7 +32,7 @@ constexpr int RS_THREADS = 256;   // rowstats block (8 independent warps)
 constexpr int RS_UNROLL = 6;      // float4 loads in flight per lane: 61 registers, 32 warps per SM (4, 8, 12, 16 measured slower)
 constexpr int SEG = 128;          // vocabulary elements per sampling segment (one warp, float4 per lane)
 constexpr int SEG_THREADS = 256;
-constexpr int MAX_SPLITS = 16;    // blocks per sequence in the sampling kernel
+constexpr int MAX_SPLITS = 64;    // blocks per sequence in the sampling kernel (small batches: enough blocks to fill the GPU)
 constexpr int MIN_SLICE = 2048;
 constexpr int MAX_SLICE = 16384;
 constexpr int MAX_GAMMA = 64;
@@ -322,12 +322,17 @@ __device__ __forceinline__ RowPartial load_partial(const RowPartial *q)
 }
 
 // ---------------------------------------------------------------------------------------------
-// Decision of one sequence (one warp): ln Z per row, ratios, first rejection; the record for
-// the sampling kernel goes to *rec_out.
+// Decision of one sequence (one block of DEC_THREADS): ln Z per row, ratios, first rejection; the
+// record for the sampling kernel goes to *rec_out.  The slice statistics of the rows are merged
+// by groups of lanes, one group per row, its lanes over the slices (a shuffle butterfly);
+// warp 0 then evaluates the positions in parallel and lane 0 walks to the first rejection.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideScratch *sc, int lane, SeqRecord *rec_out)
+constexpr int DEC_THREADS = 128;
+
+__device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideScratch *sc, int tid, SeqRecord *rec_out)
 {
     constexpr bool write = true;
+    const int lane = tid & 31, warp = tid >> 5;
     const sv_accept_params &p = a.p;
     const int gmax = p.gamma_max;
     const int rows_per_seq = 2 * gmax + 1;
@@ -341,48 +346,49 @@ __device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideS
     const int32_t *x = p.draft_tokens + p.cu_d[b];
     int32_t *out = p.out_tokens + (long long)b * (gmax + 1);
 
-    // ---- merge the slice statistics of every row this sequence has
-    for (int j = lane; j < rows_per_seq; j += 32) {
+    // ---- merge the slice statistics of every row this sequence has: groups of `lpr` lanes (a
+    // power of two covering the slices, at most a warp) take one row each
+    int lpr = 1;
+    while (lpr < 32 && lpr < a.n_slices) lpr <<= 1;
+    const int rows_per_pass = (DEC_THREADS / 32) * (32 / lpr);
+    const int sub = lane / lpr, sl = lane % lpr;
+    for (int j0 = 0; j0 < rows_per_seq; j0 += rows_per_pass) {
+        const int j = j0 + warp * (32 / lpr) + sub;
         const bool is_target = j <= gmax;
         const int i = is_target ? j : j - gmax - 1;
-        const bool have = is_target ? (i <= g) : (i < g && !greedy);
-        if (!have) continue;
+        const bool have = j < rows_per_seq && (is_target ? (i <= g) : (i < g && !greedy));
         const RowPartial *pp = a.partials + ((long long)b * rows_per_seq + j) * a.n_slices;
-        RowPartial first = load_partial(pp);
+        float ref = REF_INIT, v = -CUDART_INF_F;
+        double sum = 0.0;
+        int ix = 0x7fffffff;
+        if (have) {
+            for (int s0 = sl; s0 < a.n_slices; s0 += lpr) {
+                const RowPartial q = load_partial(pp + s0);
+                if (greedy) merge_argmax(v, ix, q.amax, q.aidx);
+                else merge_stats(ref, sum, q.ref, q.sum);
+            }
+        }
+        // rows that are absent ride along with neutral values: the shuffles need every lane
         if (greedy) {
-            float v = first.amax;
-            int ix = first.aidx;
-            for (int s0 = 1; s0 < a.n_slices; s0 += 4) {       // four records requested at once, merged in order
-                RowPartial q[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (s0 + u < a.n_slices) q[u] = load_partial(pp + s0 + u);
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (s0 + u < a.n_slices) merge_argmax(v, ix, q[u].amax, q[u].aidx);
-            }
-            sc->amax_idx[i] = ix;
+            for (int m = lpr >> 1; m > 0; m >>= 1)
+                merge_argmax(v, ix, __shfl_xor_sync(0xffffffffu, v, m), __shfl_xor_sync(0xffffffffu, ix, m));
+            if (have && sl == 0) sc->amax_idx[i] = ix;
         } else {
-            float ref = first.ref;
-            double sum = first.sum;
-            for (int s0 = 1; s0 < a.n_slices; s0 += 4) {
-                RowPartial q[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (s0 + u < a.n_slices) q[u] = load_partial(pp + s0 + u);
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (s0 + u < a.n_slices) merge_stats(ref, sum, q[u].ref, q[u].sum);
+            for (int m = lpr >> 1; m > 0; m >>= 1)
+                merge_stats(ref, sum, __shfl_xor_sync(0xffffffffu, ref, m), shfl_xor_f64(sum, m));
+            if (have && sl == 0) {
+                sc->rref[j] = ref;
+                sc->rsum[j] = sum;
+                // ln sum exp(x/T) = (ref + log2(sum)) * ln 2
+                const double lz = ((double)ref + log2(sum)) * 0.6931471805599453;
+                sc->logz[j] = lz;
+                if (is_target) { if (write && p.logZ_p != nullptr) p.logZ_p[p.cu_q[b] + i] = lz; }
+                else           { if (write && p.logZ_q != nullptr) p.logZ_q[p.cu_d[b] + i] = lz; }
             }
-            sc->rref[j] = ref;
-            sc->rsum[j] = sum;
-            // ln sum exp(x/T) = (ref + log2(sum)) * ln 2
-            const double lz = ((double)ref + log2(sum)) * 0.6931471805599453;
-            sc->logz[j] = lz;
-            if (is_target) { if (write && p.logZ_p != nullptr) p.logZ_p[p.cu_q[b] + i] = lz; }
-            else           { if (write && p.logZ_q != nullptr) p.logZ_q[p.cu_d[b] + i] = lz; }
         }
     }
+    __syncthreads();
+    if (warp != 0) return;
     if (write)
         for (int i = lane; i <= gmax; i += 32) out[i] = -1;
     __syncwarp();
@@ -456,9 +462,9 @@ __device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideS
     __syncwarp();
 }
 
-// Kernel 2: one warp per sequence takes the decision; it also clears the sequence's completion
+// Kernel 2: one block per sequence takes the decision; it also clears the sequence's completion
 // counter for kernel 3.
-__global__ void __launch_bounds__(32)
+__global__ void __launch_bounds__(DEC_THREADS)
 accept_decide_kernel(const __grid_constant__ AcceptLaunch a)
 {
     __shared__ DecideScratch s_dec;
@@ -820,7 +826,7 @@ static sv_status launch_accept(const sv_accept_params *p, void *scratch, int sli
     accept_rowstats_kernel<<<(int)(blocks_needed < cap ? blocks_needed : cap), RS_THREADS, 0, stream>>>(a);
     sv_status st = launch_check();
     if (st != SV_OK) return st;
-    accept_decide_kernel<<<p->batch, 32, 0, stream>>>(a);
+    accept_decide_kernel<<<p->batch, DEC_THREADS, 0, stream>>>(a);
     st = launch_check();
     if (st != SV_OK) return st;
     accept_sample_kernel<<<(unsigned)(splits * p->batch), SEG_THREADS, 0, stream>>>(a);

@@ -7,8 +7,8 @@
 //     logits and a single-pass online softmax sum with a power-of-two reference (float32
 //     ex2.approx exponentials accumulated in float64), warp-shuffle reduction, one record per
 //     item in the caller's workspace.
-//  2. draft_stop_decide_kernel -- one warp per sequence: merges the records of each draft
-//     position, evaluates the confidence c_i = 2^(max * log2(e)/T - ref) / sum in float64 and
+//  2. draft_stop_decide_kernel -- one block per sequence, a group of lanes per draft position
+//     with its lanes over the slice records: merges them, evaluates the confidence c_i = 2^(max * log2(e)/T - ref) / sum in float64 and
 //     takes the first position below tau.
 #include "common.cuh"
 
@@ -141,36 +141,57 @@ draft_conf_rowstats_kernel(const __grid_constant__ DraftStopLaunch a)
     }
 }
 
-__global__ void __launch_bounds__(32)
+constexpr int DSD_THREADS = 128;
+
+__global__ void __launch_bounds__(DSD_THREADS)
 draft_stop_decide_kernel(const __grid_constant__ DraftStopLaunch a)
 {
     const sv_draft_stop_params &p = a.p;
-    const int b = blockIdx.x, lane = threadIdx.x;
+    __shared__ unsigned char s_below[DS_MAX_GAMMA];
+    const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = ds_gamma(p, b);
     const float Tf = ds_temperature(p, b);
     const double tau = (double)p.tau;
+    // groups of `lpr` lanes (a power of two covering the slices, at most a warp) take one draft
+    // position each, their lanes over the slice records of its row (a shuffle butterfly)
+    int lpr = 1;
+    while (lpr < 32 && lpr < a.n_slices) lpr <<= 1;
+    const int per_pass = (DSD_THREADS / 32) * (32 / lpr);
+    const int sub = lane / lpr, sl = lane % lpr;
+    for (int i0 = 0; i0 < g; i0 += per_pass) {
+        const int i = i0 + warp * (32 / lpr) + sub;
+        const bool have = i < g;
+        double conf = 1.0;                             // greedy draft: the drafted token has probability one
+        if (Tf > 0.f) {                                // the same for the whole block
+            const ConfPartial *pp = a.partials + ((long long)b * p.gamma_max + i) * a.n_slices;
+            float ref = REF_INIT, amax = -CUDART_INF_F;
+            double sum = 0.0;
+            if (have) {
+                for (int s = sl; s < a.n_slices; s += lpr) {
+                    const ConfPartial q = pp[s];
+                    merge_stats(ref, sum, q.ref, q.sum);
+                    amax = fmaxf(amax, q.amax);
+                }
+            }
+            for (int m = lpr >> 1; m > 0; m >>= 1) {
+                merge_stats(ref, sum, __shfl_xor_sync(0xffffffffu, ref, m), shfl_xor_f64(sum, m));
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, m));
+            }
+            // top probability = exp(max/T) / sum_k exp(x_k/T) = 2^(max c - ref) / sum
+            if (have) conf = exp2((double)amax * (1.4426950408889634 / (double)Tf) - (double)ref) / sum;
+        }
+        if (have && sl == 0) {
+            if (!(conf == conf)) set_status(p.device_status, SV_DEV_NONFINITE);
+            if (p.top_prob != nullptr) p.top_prob[p.cu_d[b] + i] = conf;
+            s_below[i] = conf < tau;
+        }
+    }
+    __syncthreads();
+    if (warp != 0) return;
     int first = g;                                     // first position whose confidence is below tau
     for (int i0 = 0; i0 < g; i0 += 32) {
         const int i = i0 + lane;
-        bool below = false;
-        if (i < g) {
-            double conf = 1.0;                         // greedy draft: the drafted token has probability one
-            if (Tf > 0.f) {
-                const ConfPartial *pp = a.partials + ((long long)b * p.gamma_max + i) * a.n_slices;
-                float ref = pp[0].ref, amax = pp[0].amax;
-                double sum = pp[0].sum;
-                for (int s = 1; s < a.n_slices; ++s) {
-                    merge_stats(ref, sum, pp[s].ref, pp[s].sum);
-                    amax = fmaxf(amax, pp[s].amax);
-                }
-                // top probability = exp(max/T) / sum_k exp(x_k/T) = 2^(max c - ref) / sum
-                conf = exp2((double)amax * (1.4426950408889634 / (double)Tf) - (double)ref) / sum;
-                if (!(conf == conf)) set_status(p.device_status, SV_DEV_NONFINITE);
-            }
-            if (p.top_prob != nullptr) p.top_prob[p.cu_d[b] + i] = conf;
-            below = conf < tau;
-        }
-        const unsigned m = __ballot_sync(0xffffffffu, below);
+        const unsigned m = __ballot_sync(0xffffffffu, i < g && s_below[i] != 0);
         if (m != 0 && first == g) first = i0 + __ffs(m) - 1;
     }
     if (lane == 0) p.n_drafted[b] = first < g ? first + 1 : g;
@@ -233,6 +254,6 @@ extern "C" sv_status spec_draft_stop(const sv_draft_stop_params *p, void *worksp
         const sv_status st = sv::launch_check();
         if (st != SV_OK) return st;
     }
-    sv::draft_stop_decide_kernel<<<p->batch, 32, 0, s>>>(a);
+    sv::draft_stop_decide_kernel<<<p->batch, sv::DSD_THREADS, 0, s>>>(a);
     return sv::launch_check();
 }
