@@ -486,10 +486,18 @@ __device__ __forceinline__ void load4(const float *row, int k0, int V, bool vec,
 }
 
 // ---------------------------------------------------------------------------------------------
-// Inverse CDF of one sequence, one warp (after all blocks of the sequence have stored their sums).
+// Inverse CDF of one sequence (after all blocks of the sequence have stored their sums).  Called
+// by the whole block: all threads bring the segments' normalised masses into shared memory at
+// once (one round of loads instead of a warp's serial walk through global memory; this phase is
+// exposed when the batch is small), then warp 0 finds the segment and the token.  Rows with
+// more than PICK_SEGS segments are read in place.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const SeqRecord &rec, int lane, const double *tab)
+constexpr int PICK_SEGS = 2048;     // 2 x 16 KB of shared memory: vocabularies up to 262144
+
+__device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const SeqRecord &rec, int tid, const double *tab,
+                                         double (*s_w)[PICK_SEGS])
 {
+    const int lane = tid & 31;
     const sv_accept_params &p = a.p;
     const bool residual = rec.mode == 1;
     const int V = p.vocab, n_seg = a.n_seg, n = rec.n;
@@ -507,12 +515,23 @@ __device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const Seq
     }
     const double inv_zp = 1.0 / Zp, inv_zq = residual ? 1.0 / Zq : 0.0;
 
+    auto seg_w_global = [&](int s, bool use_r) {
+        return use_r ? __ldcg(&seg_ap[s]) * inv_zp - __ldcg(&seg_bp[s]) * inv_zq : __ldcg(&seg_a[s]) * inv_zp;
+    };
+    const bool staged = n_seg <= PICK_SEGS;
+    if (staged) {
+        for (int s = tid; s < n_seg; s += SEG_THREADS) {
+            s_w[0][s] = seg_w_global(s, false);
+            if (residual) s_w[1][s] = seg_w_global(s, true);
+        }
+    }
+    __syncthreads();
+    if (tid >= 32) return;
+    auto seg_w = [&](int s, bool use_r) { return staged ? s_w[use_r ? 1 : 0][s] : seg_w_global(s, use_r); };
+
     // total mass; lane l owns the contiguous segments [l*per, (l+1)*per)
     const int per = (n_seg + 31) / 32;
     const int s_lo = min(lane * per, n_seg), s_hi = min(s_lo + per, n_seg);
-    auto seg_w = [&](int s, bool use_r) {
-        return use_r ? __ldcg(&seg_ap[s]) * inv_zp - __ldcg(&seg_bp[s]) * inv_zq : __ldcg(&seg_a[s]) * inv_zp;
-    };
     double mine = 0.0;
     if (residual) for (int s = s_lo; s < s_hi; ++s) mine += seg_w(s, true);
     double W = warp_sum_f64(mine);
@@ -633,6 +652,7 @@ accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
     __shared__ double s_tab[128];
     __shared__ double s_red[2 * (SEG_THREADS / 32)];
     __shared__ int s_last;
+    __shared__ double s_w[2][PICK_SEGS];
     const int b = blockIdx.x / a.splits, sp = blockIdx.x % a.splits;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid >= 128) s_tab[tid - 128] = g_exp2_table[tid - 128];
@@ -729,9 +749,9 @@ accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
         s_last = atomicAdd(&a.done[b], 1u) + 1 == (unsigned)a.splits;
     }
     __syncthreads();
-    if (s_last && warp == 0) {
+    if (s_last) {             // the same for the whole block
         __threadfence();
-        pick_seq(a, b, rec, lane, s_tab);
+        pick_seq(a, b, rec, tid, s_tab, s_w);
     }
 }
 
