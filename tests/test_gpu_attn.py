@@ -55,6 +55,13 @@ def test_ragged_gqa_many_sequences():
     check_attn(make_attn_case(cfg))
 
 
+def test_many_short_sequences():
+    # far more (sequence, kv head) pairs than thread blocks, one tile each: every block's share is a
+    # run of whole pairs, and the schedule's scans run over a batch of 1500
+    cfg = synth.VerifyConfig("short", 1500, 8, 2, 128, 100, 1, 60, 0, 4, 4, 1.0, 1.0, q_scale=3.0, seed=52)
+    check_attn(make_attn_case(cfg))
+
+
 def test_mixed_row_counts_around_128():
     # 8 query heads per kv head, gamma from 0 to 16: pairs with 8 .. 136 rows in one launch,
     # so pairs that need the second row group alternate with pairs that do not
