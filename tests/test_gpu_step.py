@@ -12,11 +12,13 @@ from tests.harness import (ATTN_ATOL, DEV, AcceptOut, bits_of, compare_accept, d
 pytestmark = pytest.mark.gpu
 
 
-def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0, append=False):
+def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0, append=False, tau=None):
     """Runs `steps` verify steps on the device with padded row slabs; every per-step input is
     uploaded before the loop and nothing is read back until it ends.  Returns what the
     oracle needs to replay the same steps, and the device's logs.  With `append` every step
-    first writes that step's new keys and values behind the contexts (spec_kv_append)."""
+    first writes that step's new keys and values behind the contexts (spec_kv_append).  With `tau`
+    the draft stops early (spec_draft_stop): the step runs with n_drafted as its gamma and the
+    controller is told both."""
     B, gmax = cfg.batch, cfg.gamma_max
     cu_q, cu_d = synth.padded_offsets(B, gmax)
     n_q, n_d = int(cu_q[-1]), int(cu_d[-1])
@@ -52,22 +54,36 @@ def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0, append=False):
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     ws_a = workspace(sv.spec_verify_attn_workspace_bytes(B, gmax, cfg.hq, cfg.hkv, cfg.head_dim, max_len))
     ws_s = workspace(sv.spec_accept_sample_workspace_bytes(B, gmax, cfg.vocab))
+    ws_d = workspace(sv.spec_draft_stop_workspace_bytes(B, gmax, cfg.vocab))
+    n_dr = torch.zeros((steps, B), dtype=torch.int32, device=DEV)
     sl0 = sl.clone()
     for t in range(steps):
         tl, dl, x, ua, us, q = d_in[t]
+        gt = g                                          # the draft lengths this step runs with
+        if tau is not None:
+            # the block appended before the step has gamma + 1 positions; the step uses n_drafted + 1 of them
+            sv.spec_draft_stop(dl, cfg.temperature, tau, g, d_cd, gmax, n_dr[t], ws_d, device_status=status)
+            gt = n_dr[t]
+            sl_t = sl - g + gt                          # device arithmetic, no read-back
+        else:
+            sl_t = sl
         if append:
-            sv.spec_kv_append(d_kv[t][0], d_kv[t][1], pool, bt, sl, g, d_cq, gmax, device_status=status)
-        sv.spec_verify_attn(q, o[t], pool, bt, sl, g, d_cq, gmax, max_len, ws_a, device_status=status)
-        sv.spec_accept_sample(tl, dl, x, ua, us, cfg.temperature, g, d_cq, d_cd, gmax, n_acc, toks[t], ws_s,
+            sv.spec_kv_append(d_kv[t][0], d_kv[t][1], pool, bt, sl_t, gt, d_cq, gmax, device_status=status)
+        sv.spec_verify_attn(q, o[t], pool, bt, sl_t, gt, d_cq, gmax, max_len, ws_a, device_status=status)
+        sv.spec_accept_sample(tl, dl, x, ua, us, cfg.temperature, gt, d_cq, d_cd, gmax, n_acc, toks[t], ws_s,
                               device_status=status)
-        sv.gamma_tune_update(n_acc, gbar, g, sl, d_cq, d_cd, gcfg, trajectory=traj, accepted_log=n_log,
-                             step=t, device_status=status)
+        sv.gamma_tune_update(n_acc, gbar, g, sl_t if tau is not None else sl, d_cq, d_cd, gcfg, trajectory=traj,
+                             accepted_log=n_log, step=t, device_status=status,
+                             n_drafted=n_dr[t] if tau is not None else None)
+        if tau is not None:
+            sl = sl_t                                   # updated in place by the controller
     torch.cuda.synchronize()
     assert status.item() == 0
     return dict(kv=kv, inputs=inputs, qs=qs, cu_q=cu_q, cu_d=cu_d, sl0=sl0.cpu().numpy(),
                 toks=toks.cpu().numpy(), n_log=n_log.cpu().numpy(), traj=traj.cpu().numpy(),
                 o=o, gbar=gbar.cpu().numpy(), sl=sl.cpu().numpy(), kv_new=kv_new,
-                k_pool=bits_of(k) if append else None, v_pool=bits_of(v) if append else None)
+                k_pool=bits_of(k) if append else None, v_pool=bits_of(v) if append else None,
+                n_dr=n_dr.cpu().numpy() if tau is not None else None, tau=tau)
 
 
 def replay_with_oracle(cfg, run, steps, gamma0, gcfg, check_attn_steps=()):
@@ -79,6 +95,12 @@ def replay_with_oracle(cfg, run, steps, gamma0, gcfg, check_attn_steps=()):
     kp, vp = run["kv"].k_pool, run["kv"].v_pool
     for t in range(steps):
         li = run["inputs"][t]
+        g_issued = g
+        if run["tau"] is not None:
+            o_n, _, o_flag = oracle.draft_stop(li.draft_logits, cfg.temperature, run["tau"], g, run["cu_d"])
+            assert o_flag.any() or np.array_equal(run["n_dr"][t], o_n)
+            g = run["n_dr"][t].copy()                   # follow the device through a flagged near tie
+            sl = sl - g_issued + g
         if run["kv_new"]:
             kp, vp = oracle.kv_append(run["kv_new"][t][0], run["kv_new"][t][1], kp, vp, run["kv"].strides,
                                       run["kv"].block_table, sl, g, run["cu_q"], cfg.page_size)
@@ -94,8 +116,9 @@ def replay_with_oracle(cfg, run, steps, gamma0, gcfg, check_attn_steps=()):
                 rows = slice(run["cu_q"][b], run["cu_q"][b] + g[b] + 1)
                 assert np.abs(o_gpu[rows] - o_ref[rows]).max() <= ATTN_ATOL
         # follow the device through near ties (compare_accept has already checked legality)
-        gbar, g, sl, _, _ = oracle.gamma_tune_update(run["n_log"][t], gbar, g, sl, gcfg.eta, gcfg.delta,
-                                                     gcfg.gamma_min, gcfg.gamma_max, gcfg.mode, True)
+        gbar, g, sl, _, _ = oracle.gamma_tune_update(run["n_log"][t], gbar, g_issued, sl, gcfg.eta, gcfg.delta,
+                                                     gcfg.gamma_min, gcfg.gamma_max, gcfg.mode, True,
+                                                     n_drafted=g if run["tau"] is not None else None)
         np.testing.assert_array_equal(run["traj"][t], g)
     np.testing.assert_array_equal(run["gbar"].view(np.int64), gbar.view(np.int64))
     np.testing.assert_array_equal(run["sl"], sl)
@@ -144,6 +167,24 @@ def test_loop_that_appends_each_block_to_the_cache():
     replay_with_oracle(cfg, run, steps, 4, gcfg, check_attn_steps=(0, 7, 19))
     assert (run["n_log"] < run["traj"].max()).any()     # there were rejections to roll back
     assert (run["k_pool"] != run["kv"].k_pool).any()
+
+
+def test_loop_with_early_stop_and_cache_append():
+    # GammaTune+ over many steps: the draft stops at the first low-confidence position, the shortened block
+    # is appended, verified and accepted, and the controller keeps comparing with the gamma it issued
+    cfg = synth.scaled(synth.CONFIGS["c3"], batch=4, hq=8, hkv=2, ctx_lo=150, ctx_hi=150, vocab=3000)
+    gcfg = sv.GammaConfig(0.5, 2.0, 1, cfg.gamma_max, sv.SV_GT_PROPOSED, True)
+    steps = 16
+    # a threshold that about one draft position in seven falls below
+    cu_q, cu_d = synth.padded_offsets(cfg.batch, cfg.gamma_max)
+    full = np.full(cfg.batch, cfg.gamma_max, np.int32)
+    li0 = synth.make_logits(cfg, full, cu_q, cu_d, step=0, sigma_noise=0.4)
+    _, top, _ = oracle.draft_stop(li0.draft_logits, cfg.temperature, 0.0, full, cu_d)
+    tau = float(np.quantile(top, 0.15))
+    run = run_loop(cfg, steps, 6, gcfg, [0.4] * 4 + [2.0] * 4, 150, append=True, tau=tau)
+    replay_with_oracle(cfg, run, steps, 6, gcfg, check_attn_steps=(0, 9, 15))
+    issued = np.vstack([np.full((1, cfg.batch), 6), run["traj"][:-1]])
+    assert (run["n_dr"] < issued).any() and (run["n_dr"] == issued).any()     # some drafts stopped early, some did not
 
 
 def test_step_from_host_buffers_matches_device_calls():
