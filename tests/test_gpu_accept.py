@@ -61,6 +61,17 @@ def test_config_c5_shape_reduced_batch():
     check_accept(li, cfg.temperature, g, cu_q, cu_d, cfg.gamma_max)
 
 
+@pytest.mark.parametrize("T", [0.0, 0.8])
+def test_longest_draft_blocks(T):
+    # gamma up to the library's maximum of 64 (129 rows per sequence): the decision kernel merges the rows
+    # in several passes; small noise so that long runs of acceptances occur
+    cfg = synth.VerifyConfig("max", 5, 8, 2, 128, 9000, 100, 100, 64, 64, 64, T, 0.02, seed=71)
+    gamma = np.array([64, 1, 63, 0, 40], np.int32)
+    li, g, cu_q, cu_d = case(cfg, gamma=gamma, T=T, sigma=0.02)
+    gpu, ref, _, _ = check_accept(li, T, g, cu_q, cu_d, cfg.gamma_max)
+    assert ref.n_accepted.max() >= 8
+
+
 def test_full_size_c5_sampled_sequences():
     """The largest configuration at full size, launched as the benchmark launches it (batch 128,
     gamma 16 for every sequence, fixed row slabs): 12 sampled sequences against the oracle."""
