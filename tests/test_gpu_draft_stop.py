@@ -84,6 +84,18 @@ def test_small_and_odd_vocabularies(V):
     check(d, 1.0, float(np.median(top)), gamma, cu_d, 5)
 
 
+def test_longest_draft_blocks():
+    # gamma up to the maximum of 64 with several slices per row: the decision walks the positions in passes
+    rng = np.random.default_rng(21)
+    gamma = np.array([64, 0, 33, 64], np.int32)
+    cu_d = np.concatenate([[0], np.cumsum(gamma)]).astype(np.int32)
+    d = (rng.standard_normal((int(cu_d[-1]), 9000)) * 2.0).astype(np.float32)
+    _, top, _ = oracle.draft_stop(d, 1.0, 0.0, gamma, cu_d)
+    for q in (0.0, 0.02, 0.5):                               # never, late and early stops
+        n_gpu, n_ref, _, _ = check(d, 1.0, float(np.quantile(top, q)) if q > 0 else 0.0, gamma, cu_d, 64)
+    assert n_ref[0] < 64 and n_ref[1] == 0
+
+
 def test_row_stride_and_per_sequence_temperatures():
     rng = np.random.default_rng(11)
     gamma = np.array([4, 4, 2, 4], np.int32)
