@@ -18,7 +18,10 @@
  * General conventions
  *   - Pointers named "device" point to device memory owned by the caller; the
  *     library allocates no device memory and keeps no state between calls
- *     except registered KV-pool handles (host memory).
+ *     except registered KV-pool handles (host memory), a few per-device facts
+ *     it caches on the host (multiprocessor count, occupancy), and the one
+ *     built-in scratch array of spec_accept_sample_static with its cached
+ *     device address (see there).
  *   - "host" pointers are plain host memory (spec_verify_step_host prefers
  *     pinned memory so that its copies are asynchronous).
  *   - Every call is asynchronous on the given stream (a cudaStream_t passed as
@@ -58,10 +61,13 @@ enum {
 /* bits of the device status word */
 enum {
     SV_DEV_BAD_GAMMA = 1,   /* gamma[b] outside [0, gamma_max]: clamped */
-    SV_DEV_BAD_PAGE = 2,    /* block-table entry outside [0, n_pages): sequence skipped */
+    SV_DEV_BAD_PAGE = 2,    /* block-table entry outside [0, n_pages): attention reads that page as zeros
+                               and the outputs of that sequence are unspecified (other sequences are
+                               unaffected); the cache append skips that position */
     SV_DEV_BAD_TOKEN = 4,   /* draft token outside [0, vocab): position rejected */
     SV_DEV_NONFINITE = 8,   /* softmax sum not finite (NaN / +Inf logit): sequence emits -1 */
-    SV_DEV_TIMEOUT = 16,    /* a bounded device-side wait expired */
+    SV_DEV_TIMEOUT = 16,    /* a bounded device-side wait expired (also: a kernel found its shared
+                               memory misaligned and did nothing) */
     SV_DEV_BAD_LEN = 32     /* seq_len[b] < gamma[b]+1 or beyond the block table: sequence skipped */
 };
 
@@ -357,6 +363,18 @@ sv_status spec_verify_step_host(const sv_step_host_io *io, const sv_attn_params 
                                 const sv_accept_params *accept, void *accept_workspace,
                                 size_t accept_workspace_bytes, const sv_gamma_params *gamma,
                                 void *stream);
+
+/*
+ * Self-test of the bounded waits (no counterpart in the paper).  Every wait of
+ * the tensor-core kernels has a cycle budget; when it runs out the kernel sets
+ * SV_DEV_TIMEOUT and returns instead of hanging.  This call launches one thread
+ * block that waits, with a budget of limit_cycles (1 .. 2e9 SM cycles), on a
+ * barrier nothing ever arrives at.  Afterwards *device_status has
+ * SV_DEV_TIMEOUT set and *device_result is 0 (1 would mean the wait was
+ * satisfied); the context stays usable.
+ */
+sv_status sv_selftest_wait_expiry(uint32_t *device_status, int32_t *device_result, int64_t limit_cycles,
+                                  void *stream);
 
 /* Kernel launches issued by the library since it was loaded (for reporting). */
 uint64_t sv_launch_count(void);

@@ -26,6 +26,7 @@ EXPORTS = (
     "spec_verify_attn_workspace_bytes", "spec_verify_attn", "spec_accept_sample_workspace_bytes",
     "spec_accept_sample", "spec_accept_sample_static", "gamma_tune_update", "gamma_tune_init",
     "spec_verify_step_host", "spec_draft_stop_workspace_bytes", "spec_draft_stop", "spec_kv_append",
+    "sv_selftest_wait_expiry",
 )
 
 
@@ -125,6 +126,8 @@ def load():
         lib.gamma_tune_update.argtypes = [C.POINTER(GammaParams), C.c_void_p]
         lib.gamma_tune_init.restype = C.c_int32
         lib.gamma_tune_init.argtypes = [C.POINTER(GammaParams), C.c_int32, C.c_void_p]
+        lib.sv_selftest_wait_expiry.restype = C.c_int32
+        lib.sv_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
         lib.spec_draft_stop_workspace_bytes.restype = C.c_size_t
         lib.spec_draft_stop_workspace_bytes.argtypes = [C.c_int32] * 3
         lib.spec_draft_stop.restype = C.c_int32
@@ -458,3 +461,12 @@ def step_host_io(q_host, target_logits_host, draft_logits_host, draft_tokens_hos
     io.gamma_next_host = _host(gamma_next_host, torch.int32, "gamma_next_host")
     io.o_host = _host(o_host, torch.bfloat16, "o_host", True)
     return io
+
+
+# --------------------------------------------------------------------------- self-test
+def sv_selftest_wait_expiry(device_status, device_result, limit_cycles, stream=None):
+    """One thread block waits, with a budget of `limit_cycles`, on a barrier nothing arrives at."""
+    _check("sv_selftest_wait_expiry",
+           load().sv_selftest_wait_expiry(_dev(device_status, torch.int32, "device_status"),
+                                          _dev(device_result, torch.int32, "device_result"),
+                                          int(limit_cycles), _stream(stream)))

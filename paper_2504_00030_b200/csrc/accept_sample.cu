@@ -36,13 +36,14 @@ constexpr int MAX_SPLITS = 64;    // blocks per sequence in the sampling kernel 
 constexpr int MIN_SLICE = 2048;
 constexpr int MAX_SLICE = 16384;
 constexpr int MAX_GAMMA = 64;
+constexpr int MAX_DEVICES = 64;
 
 struct __align__(16) RowPartial {
     double sum;     // sum of 2^(x*c - ref) over the slice
     float ref;      // integer-valued reference exponent
     float amax;     // greedy rows: largest logit of the slice
     int32_t aidx;   // ... and its lowest index
-    int32_t pad;
+    int32_t bad;    // greedy rows: nonzero if the slice held a NaN (or +inf beside -inf)
 };
 
 // what the decision leaves for the sampling pass
@@ -207,7 +208,7 @@ accept_rowstats_kernel(const __grid_constant__ AcceptLaunch a)
         float ref = REF_INIT;
         double sum = 0.0;
         float amax = -CUDART_INF_F;
-        int aidx = 0x7fffffff;
+        int aidx = 0x7fffffff, bad = 0;
 
         // c = log2(e)/T split into a float pair with a strictly positive low part, so that
         // x = -inf gives -inf (never inf - inf) and NaN / +inf inputs surface in the sum.
@@ -224,6 +225,8 @@ accept_rowstats_kernel(const __grid_constant__ AcceptLaunch a)
 
         auto consume4 = [&](float x0, float x1, float x2, float x3, int k0) {
             if (greedy) {
+                const float s4 = (x0 + x1) + (x2 + x3);       // NaN if any of the four is (padding is -inf)
+                if (!(s4 == s4)) bad = 1;
                 if (x0 > amax) { amax = x0; aidx = k0; }
                 if (x1 > amax) { amax = x1; aidx = k0 + 1; }
                 if (x2 > amax) { amax = x2; aidx = k0 + 2; }
@@ -288,6 +291,7 @@ accept_rowstats_kernel(const __grid_constant__ AcceptLaunch a)
                 const int i2 = __shfl_xor_sync(0xffffffffu, aidx, m);
                 merge_argmax(amax, aidx, v2, i2);
             }
+            bad = __any_sync(0xffffffffu, bad != 0) ? 1 : 0;
         } else {
             float r = ref;
 #pragma unroll
@@ -301,7 +305,7 @@ accept_rowstats_kernel(const __grid_constant__ AcceptLaunch a)
             out.ref = ref;
             out.amax = amax;
             out.aidx = aidx;
-            out.pad = 0;
+            out.bad = bad;
             a.partials[(long long)dense_row * a.n_slices + slice_id] = out;
         }
     }
@@ -317,7 +321,7 @@ __device__ __forceinline__ RowPartial load_partial(const RowPartial *q)
     r.ref = __int_as_float(v.z);
     r.amax = __int_as_float(v.w);
     r.aidx = w.x;
-    r.pad = 0;
+    r.bad = w.y;
     return r;
 }
 
@@ -360,19 +364,22 @@ __device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideS
         const RowPartial *pp = a.partials + ((long long)b * rows_per_seq + j) * a.n_slices;
         float ref = REF_INIT, v = -CUDART_INF_F;
         double sum = 0.0;
-        int ix = 0x7fffffff;
+        int ix = 0x7fffffff, bad = 0;
         if (have) {
             for (int s0 = sl; s0 < a.n_slices; s0 += lpr) {
                 const RowPartial q = load_partial(pp + s0);
-                if (greedy) merge_argmax(v, ix, q.amax, q.aidx);
+                if (greedy) { merge_argmax(v, ix, q.amax, q.aidx); bad |= q.bad; }
                 else merge_stats(ref, sum, q.ref, q.sum);
             }
         }
         // rows that are absent ride along with neutral values: the shuffles need every lane
         if (greedy) {
-            for (int m = lpr >> 1; m > 0; m >>= 1)
+            for (int m = lpr >> 1; m > 0; m >>= 1) {
                 merge_argmax(v, ix, __shfl_xor_sync(0xffffffffu, v, m), __shfl_xor_sync(0xffffffffu, ix, m));
-            if (have && sl == 0) sc->amax_idx[i] = ix;
+                bad |= __shfl_xor_sync(0xffffffffu, bad, m);
+            }
+            // a row with a NaN or +inf logit, or with nothing above -inf, has no argmax
+            if (have && sl == 0) sc->amax_idx[i] = (bad != 0 || v == CUDART_INF_F) ? 0x7fffffff : ix;
         } else {
             for (int m = lpr >> 1; m > 0; m >>= 1)
                 merge_stats(ref, sum, __shfl_xor_sync(0xffffffffu, ref, m), shfl_xor_f64(sum, m));
@@ -403,8 +410,8 @@ __device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideS
             if (write) set_status(p.device_status, SV_DEV_BAD_TOKEN);
             code = 0;
         } else if (greedy) {
-            code = (sc->amax_idx[i] == xi) ? 1 : 0;
-            r = (double)code;
+            code = (sc->amax_idx[i] == 0x7fffffff) ? 2 : (sc->amax_idx[i] == xi) ? 1 : 0;
+            r = (code == 1) ? 1.0 : 0.0;
         } else {
             const double lzp = sc->logz[i], lzq = sc->logz[gmax + 1 + i];
             if (!(isfinite(lzp) && isfinite(lzq))) {
@@ -437,6 +444,7 @@ __device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideS
         if (write && p.ratio != nullptr)
             for (int i = n + 1; i < g; ++i) p.ratio[p.cu_d[b] + i] = CUDART_NAN;
         if (!greedy && ok && !isfinite(sc->logz[n])) ok = 0;
+        if (greedy && ok && sc->amax_idx[n] == 0x7fffffff) ok = 0;
         if (write && !ok) set_status(p.device_status, SV_DEV_NONFINITE);
         if (write && flags != 0 && p.flag_count != nullptr) atomicAdd(p.flag_count, flags);
         if (write) p.n_accepted[b] = ok ? n : 0;
@@ -834,15 +842,17 @@ static sv_status launch_accept(const sv_accept_params *p, void *scratch, int sli
 
     const long long n_items = (long long)p->batch * (2 * p->gamma_max + 1) * a.n_slices;
     const long long blocks_needed = (n_items + RS_THREADS / 32 - 1) / (RS_THREADS / 32);
-    static int blocks_per_sm = 0;       // resident blocks per SM, asked once
-    if (blocks_per_sm == 0) {
+    static int blocks_per_sm_of[MAX_DEVICES];      // resident blocks per SM, asked once per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return SV_ECUDA;
+    if (blocks_per_sm_of[dev] == 0) {
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, accept_rowstats_kernel, RS_THREADS, 0) !=
                 cudaSuccess || n < 1)
             n = 2;
-        blocks_per_sm = n;
+        blocks_per_sm_of[dev] = n;
     }
-    const long long cap = (long long)blocks_per_sm * sm_count();
+    const long long cap = (long long)blocks_per_sm_of[dev] * sm_count();
     accept_rowstats_kernel<<<(int)(blocks_needed < cap ? blocks_needed : cap), RS_THREADS, 0, stream>>>(a);
     sv_status st = launch_check();
     if (st != SV_OK) return st;
@@ -883,7 +893,6 @@ namespace sv {
 // process exits.  All calls on a device share it.
 static __device__ __align__(256) unsigned char g_accept_static_scratch[SV_ACCEPT_STATIC_SCRATCH_BYTES];
 
-constexpr int MAX_DEVICES = 64;
 static void *g_static_scratch_ptr[MAX_DEVICES];   // device address of the array, per device
 
 }  // namespace sv

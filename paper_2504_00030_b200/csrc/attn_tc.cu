@@ -26,13 +26,12 @@
 #include "tc_ptx.cuh"
 
 #include <math_constants.h>
-#include <stdlib.h>
 
 namespace sv {
 
-// Tokens per key tile are a template parameter: 64 (4 pages, 16 KB per K or V tile) when one
-// row group suffices -- two thread blocks then share an SM and hide each other's hand-off
-// latencies -- and 128 (8 pages, 32 KB) with two row groups, one block per SM.
+// This file's kernel serves pairs with 145..256 query rows (two row groups of 128, key tiles of 128
+// tokens, one block per SM); pairs with up to 144 rows go to attn_tq.cu.  Row groups and tile size
+// are template parameters.
 constexpr int QGROUP_BYTES = 128 * HD * 2;         // 32 KB: 128 query rows
 constexpr float RESCALE_THRESHOLD = 8.f;           // log2 units: P <= 2^8 before a lazy rescale
 
@@ -57,7 +56,7 @@ struct Shared {
 
 // ---------------------------------------------------------------------------- main kernel
 template <int NQ, int TILE>
-__global__ void __launch_bounds__(128 + 128 * NQ, (NQ == 1 && TILE == 64) ? 2 : 1)
+__global__ void __launch_bounds__(128 + 128 * NQ, 1)
 attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                const __grid_constant__ CUtensorMap v_map)
 {
@@ -632,8 +631,8 @@ static size_t prefix_bytes(int batch)
     return (((size_t)batch + 2 + MAX_ATTN_GRID + 1) * sizeof(int32_t) + 255) & ~(size_t)255;
 }
 
-// blocks of the main kernel: two per SM with one row group (64-token tiles), else one per SM
-static int attn_grid(int nq) { return nq == 1 ? 2 * sm_count() : sm_count(); }
+// blocks of the main kernel: one per SM
+static int attn_grid(int) { return sm_count(); }
 
 size_t attn_tc_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t hq, int32_t hkv,
                                int32_t head_dim, int32_t max_seq_len)
@@ -650,9 +649,8 @@ template <int NQ, int TILE>
 static sv_status launch_main(AttnTcLaunch &a, const sv_attn_params &p, int grid, cudaStream_t stream)
 {
     constexpr int slot_bytes = TILE * HD * 2;
-    // shared memory an SM can give to its resident blocks (1 KB per block is reserved)
-    constexpr int blocks_per_sm = (NQ == 1 && TILE == 64) ? 2 : 1;
-    const size_t budget = (228 * 1024) / blocks_per_sm - 1024;
+    // shared memory an SM can give to its one resident block (1 KB per block is reserved)
+    const size_t budget = 228 * 1024 - 1024;
     const size_t fixed = (size_t)NQ * QGROUP_BYTES + ((sizeof(Shared) + 127) & ~(size_t)127);
     a.n_slots = (int)((budget - fixed) / slot_bytes);
     if (a.n_slots > 8) a.n_slots = 8;
@@ -665,18 +663,6 @@ static sv_status launch_main(AttnTcLaunch &a, const sv_attn_params &p, int grid,
     return launch_check();
 }
 
-// 0 = pick by shape, 1 = always the shared-memory-Q kernels of this file, 2 = the
-// tensor-memory-Q kernel whenever it supports the shape.  Read once from SV_ATTN_VARIANT
-// (a diagnostic switch; both choices compute the same thing).
-static int attn_variant()
-{
-    static const int v = [] {
-        const char *e = getenv("SV_ATTN_VARIANT");
-        return (e != nullptr && e[0] >= '0' && e[0] <= '2') ? e[0] - '0' : 0;
-    }();
-    return v;
-}
-
 sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t workspace_bytes,
                          cudaStream_t stream)
 {
@@ -686,8 +672,7 @@ sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t worksp
     a.group = p.hq / p.hkv;
     a.nq = rows_groups(p);
     const int rows = a.group * (p.gamma_max + 1);
-    const int variant = attn_variant();
-    const bool use_tq = attn_tq_supported(p) && variant != 1;
+    const bool use_tq = attn_tq_supported(p);
     a.slot_rows = use_tq ? attn_tq_slot_rows(rows) : a.nq * 128;
     const int grid = use_tq ? sm_count() : attn_grid(a.nq);
     if (grid > MAX_ATTN_GRID) return SV_EUNSUPPORTED;
@@ -697,7 +682,7 @@ sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t worksp
     a.ws_part = reinterpret_cast<float *>(static_cast<uint8_t *>(workspace) + prefix_bytes(p.batch));
     sv_status st;
     if (use_tq) st = launch_attn_tq_main(a, p, grid, stream);
-    else st = a.nq == 1 ? launch_main<1, 64>(a, p, grid, stream) : launch_main<2, 128>(a, p, grid, stream);
+    else st = launch_main<2, 128>(a, p, grid, stream);
     if (st != SV_OK) return st;
     attn_combine_kernel<<<grid, COMBINE_THREADS, 0, stream>>>(a);
     return launch_check();

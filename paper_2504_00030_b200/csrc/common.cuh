@@ -21,7 +21,7 @@ inline sv_status launch_check()
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// cached per-process device facts
+// multiprocessors of the current device (cached per device)
 int sm_count();
 
 __device__ __forceinline__ void set_status(uint32_t *status, uint32_t bits)
@@ -80,12 +80,15 @@ __device__ __forceinline__ double warp_sum_f64(double v)
 // ---- online softmax statistics shared by the kernels that stream logit rows
 constexpr float REF_INIT = -1.0e30f;    // running reference before the first element
 
-// x * 2^k for k <= 0, exact (x >= 0, normal or zero); far below the reference -> 0
+// x * 2^k for k <= 0, exact while the result is a normal number (x >= 0); a result below the
+// normal range, or a shift far below the reference, gives 0
 __device__ __forceinline__ double scale_down_pow2(double x, float k)
 {
     if (!(k > -800.f) || !(x > 0.0)) return (x != x) ? x : 0.0;     // NaN stays NaN
     if (k == 0.f || x == CUDART_INF) return x;
-    return __hiloint2double(__double2hiint(x) + ((int)k << 20), __double2loint(x));
+    const int hi = __double2hiint(x);
+    if (((hi >> 20) & 0x7ff) + (int)k < 1) return 0.0;              // the exponent field would wrap
+    return __hiloint2double(hi + ((int)k << 20), __double2loint(x));
 }
 
 // (ref, sum) pairs combine by rescaling to the larger reference; the factor is a power of two.

@@ -240,14 +240,17 @@ extern "C" sv_status spec_draft_stop(const sv_draft_stop_params *p, void *worksp
     a.vec_ok = (p->row_stride % 4 == 0) && sv::aligned16(p->draft_logits);
     const long long n_items = (long long)p->batch * p->gamma_max * a.n_slices;
     if (n_items > 0) {
-        static int blocks_per_sm = 0;       // resident blocks per SM, asked once
-        if (blocks_per_sm == 0) {
+        static int blocks_per_sm_of[64];    // resident blocks per SM, asked once per device
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SV_ECUDA;
+        if (blocks_per_sm_of[dev] == 0) {
             int n = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, sv::draft_conf_rowstats_kernel, sv::DS_THREADS,
                                                               0) != cudaSuccess || n < 1)
                 n = 2;
-            blocks_per_sm = n;
+            blocks_per_sm_of[dev] = n;
         }
+        const int blocks_per_sm = blocks_per_sm_of[dev];
         const long long blocks_needed = (n_items + sv::DS_THREADS / 32 - 1) / (sv::DS_THREADS / 32);
         const long long cap = (long long)blocks_per_sm * sv::sm_count();
         sv::draft_conf_rowstats_kernel<<<(int)(blocks_needed < cap ? blocks_needed : cap), sv::DS_THREADS, 0, s>>>(a);

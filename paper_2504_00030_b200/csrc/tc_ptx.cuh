@@ -159,8 +159,10 @@ __device__ __forceinline__ uint32_t instr_desc(bool b_n_major, int n)
 }
 
 // Bounded mbarrier wait: gives up when another thread of the block has already given up or
-// after WAIT_CYCLES, sets the block's abort flag and reports SV_DEV_TIMEOUT.
-__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, int *abort_flag, uint32_t *status)
+// after `limit` cycles (WAIT_CYCLES in every kernel of the library), sets the block's abort flag
+// and reports SV_DEV_TIMEOUT.
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, int *abort_flag, uint32_t *status,
+                                             long long limit = WAIT_CYCLES)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -169,7 +171,7 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, int 
         for (int it = 0; it < 256; ++it)
             if (mbar_try_wait(bar, parity)) return true;
         if (*(volatile int *)abort_flag) return false;
-        if (clock64() - t0 > WAIT_CYCLES) break;
+        if (clock64() - t0 > limit) break;
     }
     *(volatile int *)abort_flag = 1;
     set_status(status, SV_DEV_TIMEOUT);

@@ -226,6 +226,30 @@ def test_device_status_bits():
         np.testing.assert_array_equal(gpu.out_tokens[b], ref.out_tokens[b])
 
 
+def test_greedy_rows_without_an_argmax_set_the_status_bit():
+    """T = 0: a target row that is all -inf, or holds a NaN or +inf, has no argmax.  The header promises
+    SV_DEV_NONFINITE, no accepted drafts and -1 tokens for such a sequence, and nothing else changes."""
+    cfg = synth.VerifyConfig("bad0", 5, 1, 1, 64, 4100, 32, 32, 3, 3, 3, 0.0, 0.5, seed=11)
+    li, g, cu_q, cu_d = case(cfg)
+    li.target_logits[cu_q[0] + 0, :] = -np.inf            # sequence 0: the first row is all -inf
+    li.target_logits[cu_q[1] + 2, 4097] = np.nan          # sequence 1: a NaN in its third row (last slice)
+    li.target_logits[cu_q[3] + 1, 17] = np.inf            # sequence 3: +inf in its second row
+    li.draft_tokens[cu_d[1]:cu_d[1] + 2] = np.argmax(li.target_logits[cu_q[1]:cu_q[1] + 2], axis=1)   # two accepted first
+    li.draft_tokens[cu_d[3]] = np.argmax(li.target_logits[cu_q[3]])                                     # one accepted first
+    gpu = run_accept_gpu(li, 0.0, g, cu_q, cu_d, 3)
+    assert gpu.status & sv.SV_DEV_NONFINITE
+    for b in (0, 1, 3):
+        assert gpu.n_accepted[b] == 0 and (gpu.out_tokens[b] == -1).all(), (b, gpu.out_tokens[b])
+    clean = li.target_logits.copy()
+    for b in (0, 1, 3):
+        clean[cu_q[b]:cu_q[b + 1]] = 0.0
+    ref = oracle.accept_sample(clean, li.draft_logits, li.draft_tokens, li.u_accept, li.u_sample, 0.0, g, cu_q,
+                               cu_d, 3)
+    for b in (2, 4):
+        assert gpu.n_accepted[b] == ref.n_accepted[b]
+        np.testing.assert_array_equal(gpu.out_tokens[b], ref.out_tokens[b])
+
+
 def test_host_errors():
     t = torch.zeros((4, 100), dtype=torch.float32, device=DEV)
     i32 = torch.zeros(8, dtype=torch.int32, device=DEV)
