@@ -48,9 +48,11 @@ def test_config_c3_ragged_large_vocab():
 
 
 @pytest.mark.parametrize("T", [0.0, 1.0])
-def test_config_c4_shape_reduced_batch(T):
-    cfg = synth.scaled(synth.CONFIGS["c4"], batch=16, temperature=T)
-    for sigma in (0.15, 2.5):                   # high / low acceptance regimes
+def test_config_c4_at_its_stated_size(T):
+    # batch 64, V = 32000, gamma 1..12, both acceptance regimes (noise levels from the oracle's calibration
+    # table: acceptance about 0.9 / 0.3), every sequence against the oracle
+    cfg = synth.scaled(synth.CONFIGS["c4"], temperature=T)
+    for sigma in {1.0: (0.25, 2.0), 0.0: (0.05, 1.0)}[T]:
         li, g, cu_q, cu_d = case(cfg, sigma=sigma, T=T, padded=True)
         check_accept(li, T, g, cu_q, cu_d, cfg.gamma_max)
 

@@ -29,6 +29,13 @@ def test_config_c3_shape_reduced_batch(q_scale):
     check_attn(make_attn_case(cfg))
 
 
+@pytest.mark.parametrize("q_scale", [1.0, 6.0])
+def test_config_c3_at_its_stated_size(q_scale):
+    """Llama-3.1-8B shape as the workload states it: batch 16, 32q/8kv heads, contexts 1024..8192,
+    gamma 2..10; every output row against the oracle (plain inputs, and peaky ones so the bound bites)."""
+    check_attn(make_attn_case(synth.scaled(synth.CONFIGS["c3"], q_scale=q_scale)))
+
+
 def test_config_c4_shape_reduced():
     cfg = synth.scaled(synth.CONFIGS["c4"], batch=3, hq=8, hkv=8, ctx_lo=4096, ctx_hi=4096, q_scale=4.0)
     check_attn(make_attn_case(cfg, padded=True))
@@ -161,9 +168,11 @@ def test_host_errors():
     assert e.value.status == sv.SV_EINVAL
 
 
-def test_full_size_c5_sampled_rows():
-    """The largest configuration at full size: 40 sampled (sequence, row, head) outputs."""
-    cfg = synth.CONFIGS["c5"]
+@pytest.mark.parametrize("name,q_scale", [("c5", 1.0), ("c4", 1.0), ("c4", 4.0)])
+def test_full_size_sampled_rows(name, q_scale):
+    """The two largest configurations at full size (c5: batch 128, 64q/8kv heads, contexts 512..16384, gamma 16;
+    c4: batch 64, 40 heads, context 4096, gamma 1..12): 40 sampled (sequence, row, head) outputs each."""
+    cfg = synth.scaled(synth.CONFIGS[name], q_scale=q_scale)
     case = make_attn_case(cfg)
     o_gpu, lse_gpu, status = run_attn_gpu(case)
     assert status == 0

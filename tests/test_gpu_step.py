@@ -12,13 +12,15 @@ from tests.harness import (ATTN_ATOL, DEV, AcceptOut, bits_of, compare_accept, d
 pytestmark = pytest.mark.gpu
 
 
-def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0, append=False, tau=None):
+def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0, append=False, tau=None, n_inputs=None):
     """Runs `steps` verify steps on the device with padded row slabs; every per-step input is
     uploaded before the loop and nothing is read back until it ends.  Returns what the
     oracle needs to replay the same steps, and the device's logs.  With `append` every step
     first writes that step's new keys and values behind the contexts (spec_kv_append).  With `tau`
     the draft stops early (spec_draft_stop): the step runs with n_drafted as its gamma and the
-    controller is told both."""
+    controller is told both.  Step t draws its noise level from sigmas[t % len(sigmas)].  With
+    `n_inputs` only that many distinct input sets are generated per noise level and step t uses set
+    t % n_inputs of its level (long runs at full size: the inputs recur, the controller's state does not)."""
     B, gmax = cfg.batch, cfg.gamma_max
     cu_q, cu_d = synth.padded_offsets(B, gmax)
     n_q, n_d = int(cu_q[-1]), int(cu_d[-1])
@@ -29,16 +31,35 @@ def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0, append=False, tau=None):
     bt = dev(kv.block_table)
     max_len = L0 + steps * (gmax + 1)
     full_gamma = np.full(B, gmax, np.int32)
-    inputs = [synth.make_logits(cfg, full_gamma, cu_q, cu_d, step=t, sigma_noise=sigmas[t % len(sigmas)])
-              for t in range(steps)]
-    qs = [synth.make_q(cfg, n_q, step=t) for t in range(steps)]
+    made, made_q = {}, {}
+
+    def input_set(t):
+        key = (sigmas[t % len(sigmas)], t if n_inputs is None else t % n_inputs)
+        if key not in made:
+            made[key] = synth.make_logits(cfg, full_gamma, cu_q, cu_d, step=key[1], sigma_noise=key[0])
+        return made[key]
+
+    def q_set(t):
+        k = t if n_inputs is None else t % n_inputs
+        if k not in made_q:
+            made_q[k] = synth.make_q(cfg, n_q, step=k)
+        return made_q[k]
+
+    inputs = [input_set(t) for t in range(steps)]
+    qs = [q_set(t) for t in range(steps)]
     n_kv = n_q * cfg.hkv * cfg.head_dim
     kv_new = [(synth.normal_bf16_bits(cfg.seed, 90, n_kv, 1.0, t).reshape(n_q, cfg.hkv, cfg.head_dim),
                synth.normal_bf16_bits(cfg.seed, 91, n_kv, 1.0, t).reshape(n_q, cfg.hkv, cfg.head_dim))
               for t in range(steps)] if append else []
     d_kv = [(dev_bf16(a), dev_bf16(b)) for a, b in kv_new]
-    d_in = [(dev(li.target_logits), dev(li.draft_logits), dev(li.draft_tokens), dev(li.u_accept),
-             dev(li.u_sample), dev_bf16(q)) for li, q in zip(inputs, qs)]
+    up, up_q = {}, {}                                   # one device copy per distinct input set
+    for li, q in zip(inputs, qs):
+        if id(li) not in up:
+            up[id(li)] = (dev(li.target_logits), dev(li.draft_logits), dev(li.draft_tokens), dev(li.u_accept),
+                          dev(li.u_sample))
+        if id(q) not in up_q:
+            up_q[id(q)] = dev_bf16(q)
+    d_in = [up[id(li)] + (up_q[id(q)],) for li, q in zip(inputs, qs)]
 
     gbar = torch.zeros(B, dtype=torch.float64, device=DEV)
     g = torch.zeros(B, dtype=torch.int32, device=DEV)
@@ -86,7 +107,9 @@ def run_loop(cfg, steps, gamma0, gcfg, sigmas, L0, append=False, tau=None):
                 n_dr=n_dr.cpu().numpy() if tau is not None else None, tau=tau)
 
 
-def replay_with_oracle(cfg, run, steps, gamma0, gcfg, check_attn_steps=()):
+def replay_with_oracle(cfg, run, steps, gamma0, gcfg, check_attn_steps=(), attn_samples=None):
+    """The oracle takes the same steps.  At `check_attn_steps` the attention outputs are compared too:
+    every row, or with `attn_samples` that many seeded (sequence, row, head) outputs computed one by one."""
     B, gmax = cfg.batch, cfg.gamma_max
     gbar, g, _, _ = oracle.gamma_tune_init(B, gamma0, gmax, True)
     sl = run["sl0"].copy()
@@ -107,7 +130,18 @@ def replay_with_oracle(cfg, run, steps, gamma0, gcfg, check_attn_steps=()):
         gpu = AcceptOut(run["n_log"][t], run["toks"][t], None, None, None, 0, 0)
         ref, n_pos, n_tok = compare_accept(gpu, li, cfg.temperature, g, run["cu_q"], run["cu_d"], gmax)
         flagged += n_pos + n_tok
-        if t in check_attn_steps:
+        if t in check_attn_steps and attn_samples is not None:
+            o_gpu = synth.bf16_to_f32(bits_of(run["o"][t])).astype(np.float64)
+            rng = np.random.default_rng(1000 + t)
+            for _ in range(attn_samples):
+                b = int(rng.integers(B))
+                i = int(rng.integers(g[b] + 1))
+                h = int(rng.integers(cfg.hq))
+                row = run["cu_q"][b] + i
+                o_ref, _ = oracle.attn_row(run["qs"][t][row, h], kp, vp, run["kv"].strides, run["kv"].block_table[b],
+                                           cfg.page_size, h // cfg.group, int(sl[b]) - (int(g[b]) + 1) + i + 1, scale)
+                assert np.abs(o_gpu[row, h] - o_ref).max() <= ATTN_ATOL
+        elif t in check_attn_steps:
             o_ref, _ = oracle.verify_attn(run["qs"][t], kp, vp, run["kv"].strides,
                                           run["kv"].block_table, sl, g, run["cu_q"], cfg.hq, cfg.hkv,
                                           cfg.page_size, scale)
@@ -142,18 +176,61 @@ def test_c2_gamma_trajectory_device_resident(gamma0):
     assert len(np.unique(run["traj"])) >= 3            # the controller really moved gamma
 
 
+@pytest.mark.parametrize("sigma", [0.3, 1.0, 2.0])
+@pytest.mark.parametrize("gamma0", [1, 4, 8])
+def test_c2_at_its_stated_size(sigma, gamma0):
+    """vicuna-7B shape as the workload states it: 512 controller-driven steps from a 2048-token context, one run
+    per noise level and initial gamma.  Counts, tokens and trajectories are replayed by the oracle at every
+    step, the attention outputs at four of them (the context has grown by then).  The per-step inputs recur
+    every 64 steps."""
+    cfg = synth.scaled(synth.CONFIGS["c2"], ctx_lo=2048, ctx_hi=2048)
+    gcfg = sv.GammaConfig(0.5, 2.0, 1, 8, sv.SV_GT_PROPOSED, True)
+    steps = 512
+    run = run_loop(cfg, steps, gamma0, gcfg, [sigma], 2048, n_inputs=64)
+    replay_with_oracle(cfg, run, steps, gamma0, gcfg, check_attn_steps=(0, 100, 300, 511))
+    assert run["traj"].min() >= 1 and run["traj"].max() <= 8
+    mean_gamma = run["traj"][64:].mean()
+    # more noise, fewer accepted drafts, shorter blocks (the oracle's calibration: alpha 0.88 / 0.62 / 0.32)
+    assert {0.3: mean_gamma > 3.0, 1.0: 1.5 < mean_gamma < 3.5, 2.0: mean_gamma < 2.0}[sigma], mean_gamma
+
+
+# noise levels of the two acceptance regimes, from the oracle's calibration table (oracle/calibrate_sigma.py):
+# acceptance about 0.9 / about 0.3 at T = 1 (mean sum min(p, q)) and at T = 0 (greedy match rate)
+C4_SIGMA = {1.0: (0.25, 2.0), 0.0: (0.05, 1.0)}
+
+
 @pytest.mark.parametrize("T", [0.0, 1.0])
 def test_c4_alternating_regimes_reduced(T):
     # vicuna-13B shape at reduced batch / heads / context; acceptance regime flips every 8 steps
     cfg = synth.scaled(synth.CONFIGS["c4"], batch=8, hq=4, hkv=4, ctx_lo=600, ctx_hi=600, temperature=T)
     gcfg = sv.GammaConfig(0.5, 2.0, 1, 12, sv.SV_GT_PROPOSED, True)
     steps = 32
-    sig = [0.1] * 8 + [3.0] * 8
+    hi, lo = C4_SIGMA[T]
+    sig = [hi] * 8 + [lo] * 8
     run = run_loop(cfg, steps, 4, gcfg, sig, 600)
     replay_with_oracle(cfg, run, steps, 4, gcfg, check_attn_steps=(5, 20))
     easy = run["traj"][4:8].mean()
     hard = run["traj"][12:16].mean()
     assert easy > hard                                  # expands when drafts are accepted, contracts otherwise
+
+
+@pytest.mark.parametrize("T", [0.0, 1.0])
+def test_c4_at_its_stated_size(T):
+    """vicuna-13B shape as the workload states it: batch 64, 40 heads, 4096-token contexts, gamma in [1, 12]
+    driven by the controller for 256 steps, acceptance regimes of about 0.9 and about 0.3 alternating every 64
+    steps, greedy and sampling.  Every step's counts, tokens and gammas are replayed by the oracle; attention
+    outputs are compared on sampled rows in both regimes.  Eight distinct input sets per regime recur."""
+    cfg = synth.scaled(synth.CONFIGS["c4"], temperature=T)
+    gcfg = sv.GammaConfig(0.5, 2.0, 1, 12, sv.SV_GT_PROPOSED, True)
+    steps = 256
+    hi, lo = C4_SIGMA[T]
+    sig = [hi] * 64 + [lo] * 64
+    run = run_loop(cfg, steps, 4, gcfg, sig, 4096, n_inputs=8)
+    replay_with_oracle(cfg, run, steps, 4, gcfg, check_attn_steps=(3, 70, 255), attn_samples=24)
+    acc = run["n_log"].astype(np.float64) / np.maximum(np.vstack([np.full((1, cfg.batch), 4), run["traj"][:-1]]), 1)
+    easy, hard = run["traj"][32:64].mean(), run["traj"][96:128].mean()
+    assert easy > hard + 2.0, (easy, hard)              # long blocks while drafts are accepted, short ones otherwise
+    assert acc[32:64].mean() > acc[96:128].mean()
 
 
 def test_loop_that_appends_each_block_to_the_cache():
