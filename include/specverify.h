@@ -164,6 +164,36 @@ typedef struct sv_kv_append_params {
 
 sv_status spec_kv_append(const sv_kv_append_params *p, void *stream);
 
+/* ---------------------------------------------------------------- all layers of a step */
+/*
+ * A target model keeps one KV cache per layer (KV caching, paper Section 5), all
+ * with the same paging: one block table, one set of lengths.  This call runs the
+ * cache append and the verify attention of n_layers caches in one enqueue: first
+ * ONE launch writes every layer's new keys and values (spec_kv_append for all
+ * layers at once; skipped when k_new is NULL), then the attention of layer 0, 1,
+ * ... in order, each reading its own pool, queries and writing its own output.
+ * In a real model layer l+1's queries depend on layer l's output through the
+ * projections in between, which are outside this library; here they are inputs.
+ * pools / q / o / k_new / v_new / lse are HOST arrays of n_layers entries
+ * (device pointers inside); everything else is shared and means what it means in
+ * sv_attn_params.  The workspace is the one spec_verify_attn asks for (it is
+ * reused layer after layer).  Errors: as spec_verify_attn / spec_kv_append; the
+ * pools must agree in hkv and head_dim.
+ */
+typedef struct sv_attn_layers_params {
+    int32_t n_layers;
+    const sv_kv_pool_t *pools;    /* host [n_layers] */
+    const void *const *q;         /* host [n_layers] of device bf16 [n_rows, hq, head_dim] */
+    void *const *o;               /* host [n_layers] of device bf16 [n_rows, hq, head_dim] */
+    float *const *lse;            /* host [n_layers] of device fp32 [n_rows, hq], or NULL */
+    const void *const *k_new;     /* host [n_layers] of device bf16 [n_rows, hkv, head_dim], or NULL: no append */
+    const void *const *v_new;     /* host [n_layers], NULL exactly when k_new is */
+    sv_attn_params shared;        /* q, o, lse and pool of this struct are ignored */
+} sv_attn_layers_params;
+
+sv_status spec_verify_attn_layers(const sv_attn_layers_params *p, void *workspace_device,
+                                  size_t workspace_bytes, void *stream);
+
 /* ---------------------------------------------------------------- accept / resample */
 /*
  * Speculative sampling (paper Section 3, after Leviathan et al. and Chen et

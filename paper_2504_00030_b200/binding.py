@@ -26,7 +26,7 @@ EXPORTS = (
     "spec_verify_attn_workspace_bytes", "spec_verify_attn", "spec_accept_sample_workspace_bytes",
     "spec_accept_sample", "spec_accept_sample_static", "gamma_tune_update", "gamma_tune_init",
     "spec_verify_step_host", "spec_draft_stop_workspace_bytes", "spec_draft_stop", "spec_kv_append",
-    "sv_selftest_wait_expiry",
+    "sv_selftest_wait_expiry", "spec_verify_attn_layers",
 )
 
 
@@ -43,6 +43,12 @@ class AttnParams(C.Structure):
                 ("batch", C.c_int32), ("gamma_max", C.c_int32), ("hq", C.c_int32),
                 ("hkv", C.c_int32), ("head_dim", C.c_int32), ("max_seq_len", C.c_int32),
                 ("sm_scale", C.c_float), ("device_status", C.c_void_p)]
+
+
+class AttnLayersParams(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("pools", C.POINTER(C.c_void_p)), ("q", C.POINTER(C.c_void_p)),
+                ("o", C.POINTER(C.c_void_p)), ("lse", C.POINTER(C.c_void_p)), ("k_new", C.POINTER(C.c_void_p)),
+                ("v_new", C.POINTER(C.c_void_p)), ("shared", AttnParams)]
 
 
 class KvAppendParams(C.Structure):
@@ -126,6 +132,8 @@ def load():
         lib.gamma_tune_update.argtypes = [C.POINTER(GammaParams), C.c_void_p]
         lib.gamma_tune_init.restype = C.c_int32
         lib.gamma_tune_init.argtypes = [C.POINTER(GammaParams), C.c_int32, C.c_void_p]
+        lib.spec_verify_attn_layers.restype = C.c_int32
+        lib.spec_verify_attn_layers.argtypes = [C.POINTER(AttnLayersParams), C.c_void_p, C.c_size_t, C.c_void_p]
         lib.sv_selftest_wait_expiry.restype = C.c_int32
         lib.sv_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
         lib.spec_draft_stop_workspace_bytes.restype = C.c_size_t
@@ -461,6 +469,47 @@ def step_host_io(q_host, target_logits_host, draft_logits_host, draft_tokens_hos
     io.gamma_next_host = _host(gamma_next_host, torch.int32, "gamma_next_host")
     io.o_host = _host(o_host, torch.bfloat16, "o_host", True)
     return io
+
+
+# --------------------------------------------------------------------------- all layers of a step
+def attn_layers_params(qs, os_, pools, block_table, seq_len, gamma, cu_q, gamma_max, max_seq_len, k_new=None,
+                       v_new=None, lses=None, sm_scale=None, device_status=None) -> AttnLayersParams:
+    """Arguments of spec_verify_attn_layers: lists with one entry per layer, the rest shared.  The returned
+    struct keeps the pointer arrays alive."""
+    n = len(pools)
+    if not (len(qs) == n and len(os_) == n):
+        raise ValueError("one q, o and pool per layer")
+    p = AttnLayersParams()
+    p.n_layers = n
+    p.shared = attn_params(qs[0], os_[0], pools[0], block_table, seq_len, gamma, cu_q, gamma_max, max_seq_len,
+                           sm_scale, None, device_status)
+
+    def arr(ptrs):
+        a = (C.c_void_p * n)(*ptrs)
+        return a
+
+    p._keep = [arr([pl.handle.value for pl in pools]), arr([_dev(t, torch.bfloat16, "q") for t in qs]),
+               arr([_dev(t, torch.bfloat16, "o") for t in os_])]
+    p.pools, p.q, p.o = (C.cast(a, C.POINTER(C.c_void_p)) for a in p._keep)
+    if lses is not None:
+        a = arr([_dev(t, torch.float32, "lse") for t in lses])
+        p._keep.append(a)
+        p.lse = C.cast(a, C.POINTER(C.c_void_p))
+    if k_new is not None:
+        ak = arr([_dev(t, torch.bfloat16, "k_new") for t in k_new])
+        av = arr([_dev(t, torch.bfloat16, "v_new") for t in v_new])
+        p._keep += [ak, av]
+        p.k_new, p.v_new = C.cast(ak, C.POINTER(C.c_void_p)), C.cast(av, C.POINTER(C.c_void_p))
+    return p
+
+
+def spec_verify_attn_layers(qs, os_, pools, block_table, seq_len, gamma, cu_q, gamma_max, max_seq_len, workspace,
+                            k_new=None, v_new=None, lses=None, sm_scale=None, device_status=None, stream=None):
+    """Cache append (one launch for all layers) and verify attention of every layer's cache (asynchronous)."""
+    p = attn_layers_params(qs, os_, pools, block_table, seq_len, gamma, cu_q, gamma_max, max_seq_len, k_new, v_new,
+                           lses, sm_scale, device_status)
+    _check("spec_verify_attn_layers",
+           load().spec_verify_attn_layers(C.byref(p), workspace.data_ptr(), _nbytes(workspace), _stream(stream)))
 
 
 # --------------------------------------------------------------------------- self-test

@@ -163,6 +163,50 @@ extern "C" sv_status spec_verify_attn(const sv_attn_params *p, void *workspace,
     return sv::launch_attn_simple(*p, (cudaStream_t)stream);
 }
 
+extern "C" sv_status spec_verify_attn_layers(const sv_attn_layers_params *p, void *workspace,
+                                             size_t workspace_bytes, void *stream)
+{
+    if (p == nullptr || p->n_layers <= 0 || p->pools == nullptr || p->q == nullptr || p->o == nullptr)
+        return SV_EINVAL;
+    if ((p->k_new == nullptr) != (p->v_new == nullptr)) return SV_EINVAL;
+    // every layer's arguments are checked before anything is launched
+    for (int l = 0; l < p->n_layers; ++l) {
+        sv_attn_params a = p->shared;
+        a.pool = p->pools[l];
+        a.q = p->q[l];
+        a.o = p->o[l];
+        a.lse = p->lse != nullptr ? p->lse[l] : nullptr;
+        const sv_status st = check_attn(&a);
+        if (st != SV_OK) return st;
+        if (a.pool->hkv != p->pools[0]->hkv || a.pool->head_dim != p->pools[0]->head_dim) return SV_EINVAL;
+    }
+    if (p->k_new != nullptr) {
+        sv_kv_append_params ka;
+        memset(&ka, 0, sizeof ka);
+        ka.block_table = p->shared.block_table;
+        ka.block_table_stride = p->shared.block_table_stride;
+        ka.seq_len = p->shared.seq_len;
+        ka.gamma = p->shared.gamma;
+        ka.cu_q = p->shared.cu_q;
+        ka.batch = p->shared.batch;
+        ka.gamma_max = p->shared.gamma_max;
+        ka.device_status = p->shared.device_status;
+        const sv_status st = sv::launch_kv_append_layers(ka, p->pools, p->k_new, p->v_new, p->n_layers,
+                                                         (cudaStream_t)stream);
+        if (st != SV_OK) return st;
+    }
+    for (int l = 0; l < p->n_layers; ++l) {
+        sv_attn_params a = p->shared;
+        a.pool = p->pools[l];
+        a.q = p->q[l];
+        a.o = p->o[l];
+        a.lse = p->lse != nullptr ? p->lse[l] : nullptr;
+        const sv_status st = spec_verify_attn(&a, workspace, workspace_bytes, stream);
+        if (st != SV_OK) return st;
+    }
+    return SV_OK;
+}
+
 extern "C" sv_status spec_verify_step_host(const sv_step_host_io *io, const sv_attn_params *attn,
                                            void *attn_ws, size_t attn_ws_bytes,
                                            const sv_accept_params *acc, void *acc_ws,

@@ -29,4 +29,8 @@ size_t attn_tc_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t hq, int
 sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t workspace_bytes,
                          cudaStream_t stream);
 
+// The draft block's keys and values written into n caches that share one block table (kv_append.cu).
+sv_status launch_kv_append_layers(const sv_kv_append_params &shared, const sv_kv_pool_t *pools, const void *const *k_new,
+                                  const void *const *v_new, int n_layers, cudaStream_t stream);
+
 }  // namespace sv

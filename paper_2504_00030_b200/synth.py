@@ -21,7 +21,7 @@ PAGE_SIZE = 16
 _CHUNK = 1 << 22
 
 # tensor ids for the Philox key
-_T_K, _T_V, _T_Q, _T_BASE, _T_NOISE, _T_GUMBEL, _T_UACC, _T_USAMP, _T_PERM, _T_LEN, _T_GAMMA = range(11)
+_T_K, _T_V, _T_Q, _T_BASE, _T_NOISE, _T_GUMBEL, _T_UACC, _T_USAMP, _T_PERM, _T_LEN, _T_GAMMA, _T_MIX = range(12)
 
 
 def _rng(seed: int, tensor: int, chunk: int = 0, step: int = 0) -> np.random.Generator:
@@ -212,22 +212,44 @@ class LogitInputs:
     u_sample: np.ndarray        # float32 [B]
 
 
+def mixture_rows(cfg: VerifyConfig, n_rows: int, step: int, hard_prob: float,
+                 easy=(3.0, 0.3), hard=(1.0, 2.0)):
+    """Per-row (sigma_draft, sigma_noise) for a workload whose positions differ in difficulty.
+
+    Every row is "hard" with probability hard_prob (seeded) and "easy" otherwise.  An easy
+    position has a peaked draft distribution (large logit spread) that the target nearly
+    shares (small noise); a hard one a flat draft distribution far from the target's.  This
+    models the premise of confidence-guided drafting (paper Section 4.2): where the draft
+    model is unsure, its token is likely to be rejected.  Returns two float32 arrays [n_rows]."""
+    is_hard = _rng(cfg.seed, _T_MIX, 0, step).random(n_rows) < hard_prob
+    sd = np.where(is_hard, hard[0], easy[0]).astype(np.float32)
+    sn = np.where(is_hard, hard[1], easy[1]).astype(np.float32)
+    return sd, sn
+
+
 def make_logits(cfg: VerifyConfig, gamma: np.ndarray, cu_q: np.ndarray, cu_d: np.ndarray,
                 step: int = 0, sigma_noise: float | None = None,
-                temperature: float | None = None) -> LogitInputs:
+                temperature: float | None = None, row_sigmas=None) -> LogitInputs:
     """Draft logits ~N(0, sigma_draft^2), target = draft + N(0, sigma_noise^2).
 
     Rows follow cu_q / cu_d (packed or padded); rows a sequence does not use
     are still filled.  Draft tokens are exact draws from softmax(draft/T) by
     the Gumbel-max construction (argmax of draft/T + Gumbel noise) for T > 0
-    and the plain argmax for T == 0.
+    and the plain argmax for T == 0.  With row_sigmas = (sigma_draft [n_q],
+    sigma_noise [n_q]) every target row (and the draft row of the same
+    position) has its own two standard deviations (see mixture_rows).
     """
     V = cfg.vocab
     sig = cfg.sigma_noise if sigma_noise is None else sigma_noise
     T = cfg.temperature if temperature is None else temperature
     n_q, n_d = int(cu_q[-1]), int(cu_d[-1])
-    base = normal_f32(cfg.seed, _T_BASE, n_q * V, cfg.sigma_draft, step).reshape(n_q, V)
-    noise = normal_f32(cfg.seed, _T_NOISE, n_q * V, sig, step).reshape(n_q, V)
+    if row_sigmas is None:
+        base = normal_f32(cfg.seed, _T_BASE, n_q * V, cfg.sigma_draft, step).reshape(n_q, V)
+        noise = normal_f32(cfg.seed, _T_NOISE, n_q * V, sig, step).reshape(n_q, V)
+    else:
+        sd, sn = row_sigmas
+        base = normal_f32(cfg.seed, _T_BASE, n_q * V, 1.0, step).reshape(n_q, V) * np.asarray(sd, np.float32)[:, None]
+        noise = normal_f32(cfg.seed, _T_NOISE, n_q * V, 1.0, step).reshape(n_q, V) * np.asarray(sn, np.float32)[:, None]
     target = base + noise
     draft = np.empty((max(n_d, 1), V), np.float32)[:n_d]
     for b in range(len(gamma)):
