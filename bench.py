@@ -454,6 +454,18 @@ def run_ours(args):
     t_ds = median_us(lambda: check(lib.spec_draft_stop(C.byref(dp), ws_d.data_ptr(), ws_d.numel(), sptr), "draft_stop"))
     ds_bytes = int(gamma.sum()) * cfg.vocab * 4
 
+    # ---- accept / resample with the logits stored as bf16 (not part of the step above): same call, half the bytes
+    tl16, dl16 = vs.tl.to(torch.bfloat16), vs.dl.to(torch.bfloat16)
+    n16 = torch.zeros(B, dtype=torch.int32, device=DEV)
+    tok16 = torch.zeros((B, gmax + 1), dtype=torch.int32, device=DEV)
+    sp16 = sv.accept_params(tl16, dl16, vs.x, vs.ua, vs.us, cfg.temperature, vs.g, vs.cq, vs.cd, gmax, n16, tok16,
+                            device_status=status)
+    state.copy_(state0)
+    t_a16 = median_us(lambda: check(lib.spec_accept_sample(C.byref(sp16), vs.ws_s.data_ptr(), vs.ws_s.numel(), sptr),
+                                    "accept bf16"))
+    a16_bytes = synth.algorithmic_bytes(cfg, seq_len, gamma)[1] // 2
+    del tl16, dl16
+
     # ---- cache append (not part of the step above): the block's keys and values written behind the contexts
     n_kv = n_q * cfg.hkv * cfg.head_dim
     k_new = vs.up_bf16(synth.normal_bf16_bits(cfg.seed, 90, n_kv).reshape(n_q, cfg.hkv, cfg.head_dim))
@@ -544,6 +556,9 @@ def run_ours(args):
     if clocks is not None and clocks.get("sm_mhz"):
         # the GPUs of a pool differ in the clock they hold; time x clock compares kernels across them
         line["step_us_x_sm_ghz"] = 1e3 * ms_step * clocks["sm_mhz"] / 1e3
+    line["accept_bf16_logits"] = {"what": "spec_accept_sample on the same logits stored as bf16, outside the timed step",
+                                  "us": t_a16, "bytes": a16_bytes, "gbs": a16_bytes / (t_a16 * 1e-6) / 1e9,
+                                  "frac_of_measured": a16_bytes / (t_a16 * 1e-6) / 1e9 / peak}
     line["kv_append"] = {"what": "the block's keys and values written into the paged cache, outside the timed step",
                          "us": t_ka, "bytes": ka_bytes}
     if layers is not None:

@@ -210,6 +210,9 @@ sv_status spec_verify_attn_layers(const sv_attn_layers_params *p, void *workspac
  *           next = argmax(t_n); draft logits and uniforms are not read.
  * Softmax sums are accumulated in float64 from float32 exponentials; the
  * ratio, the comparison and the sampled row are evaluated in float64.
+ * The paper's largest target runs with reduced precision (Section 5); logits
+ * stored as bf16 are accepted too (logits_bf16), which halves the bytes of
+ * this step.
  */
 typedef struct sv_accept_params {
     const float *target_logits;   /* device fp32 [n_q_rows, row_stride] */
@@ -234,6 +237,12 @@ typedef struct sv_accept_params {
     double *logZ_q;               /* device out [n_d_rows] or NULL: ln sum exp(d/T) */
     uint32_t *flag_count;         /* device, one word or NULL: += positions with |u - ratio| < 1e-6 */
     uint32_t *device_status;      /* device, one word or NULL */
+    int32_t logits_bf16;          /* 0: the logits are float32 (as declared).  1: target_logits / draft_logits
+                                     point to bf16 values (2 bytes each, row_stride still in elements; a
+                                     multiple of 8 with 16-byte aligned bases enables 128-bit loads); every
+                                     value is widened exactly to float32 and the arithmetic is unchanged, so
+                                     the result is that of the float32 call on the widened values at half
+                                     the bytes */
 } sv_accept_params;
 
 size_t spec_accept_sample_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t vocab);
@@ -354,6 +363,7 @@ typedef struct sv_draft_stop_params {
     int32_t *n_drafted;           /* device out [batch] */
     double *top_prob;             /* device out [n_d_rows] or NULL: c_i of every draft row */
     uint32_t *device_status;      /* device, one word or NULL */
+    int32_t logits_bf16;          /* as in sv_accept_params: 1 = draft_logits holds bf16 values */
 } sv_draft_stop_params;
 
 size_t spec_draft_stop_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t vocab);

@@ -66,7 +66,7 @@ class AcceptParams(C.Structure):
                 ("cu_d", C.c_void_p), ("batch", C.c_int32), ("gamma_max", C.c_int32),
                 ("n_accepted", C.c_void_p), ("out_tokens", C.c_void_p), ("ratio", C.c_void_p),
                 ("logZ_p", C.c_void_p), ("logZ_q", C.c_void_p), ("flag_count", C.c_void_p),
-                ("device_status", C.c_void_p)]
+                ("device_status", C.c_void_p), ("logits_bf16", C.c_int32)]
 
 
 class GammaConfigC(C.Structure):
@@ -86,7 +86,8 @@ class DraftStopParams(C.Structure):
     _fields_ = [("draft_logits", C.c_void_p), ("row_stride", C.c_int64), ("vocab", C.c_int32),
                 ("temperature", C.c_float), ("temperature_per_seq", C.c_void_p), ("tau", C.c_float),
                 ("gamma", C.c_void_p), ("cu_d", C.c_void_p), ("batch", C.c_int32), ("gamma_max", C.c_int32),
-                ("n_drafted", C.c_void_p), ("top_prob", C.c_void_p), ("device_status", C.c_void_p)]
+                ("n_drafted", C.c_void_p), ("top_prob", C.c_void_p), ("device_status", C.c_void_p),
+                ("logits_bf16", C.c_int32)]
 
 
 class StepHostIO(C.Structure):
@@ -311,8 +312,10 @@ def accept_params(target_logits, draft_logits, draft_tokens, u_accept, u_sample,
                   logZ_q=None, flag_count=None, device_status=None,
                   temperature_per_seq=None) -> AcceptParams:
     p = AcceptParams()
-    p.target_logits = _dev(target_logits, torch.float32, "target_logits")
-    p.draft_logits = _dev(draft_logits, torch.float32, "draft_logits", True)
+    ldt = target_logits.dtype if target_logits.dtype == torch.bfloat16 else torch.float32     # float32 or bf16 logits
+    p.logits_bf16 = int(ldt == torch.bfloat16)
+    p.target_logits = _dev(target_logits, ldt, "target_logits")
+    p.draft_logits = _dev(draft_logits, ldt, "draft_logits", True)
     p.row_stride = target_logits.stride(0)
     p.vocab = target_logits.shape[-1]
     p.draft_tokens = _dev(draft_tokens, torch.int32, "draft_tokens", True)
@@ -412,7 +415,9 @@ def spec_draft_stop_workspace_bytes(batch, gamma_max, vocab) -> int:
 def draft_stop_params(draft_logits, temperature, tau, gamma, cu_d, gamma_max, n_drafted, top_prob=None,
                       device_status=None, temperature_per_seq=None) -> DraftStopParams:
     p = DraftStopParams()
-    p.draft_logits = _dev(draft_logits, torch.float32, "draft_logits")
+    ldt = draft_logits.dtype if draft_logits.dtype == torch.bfloat16 else torch.float32       # float32 or bf16 logits
+    p.logits_bf16 = int(ldt == torch.bfloat16)
+    p.draft_logits = _dev(draft_logits, ldt, "draft_logits")
     p.row_stride = draft_logits.stride(0)
     p.vocab = draft_logits.shape[-1]
     p.temperature = float(temperature)

@@ -23,6 +23,7 @@
 // fetched through an instruction cache that the streaming loop owns, under a saturated
 // memory system -- the decision alone then costs more than the whole kernel 2 and 3.)
 #include "common.cuh"
+#include "row_stream.cuh"
 
 #include <math_constants.h>
 
@@ -175,6 +176,7 @@ __device__ __forceinline__ void exp2_f64_n(const double (&y)[N], double (&out)[N
 // Dense row numbering: sequence b owns rows b*(2*gmax+1) + j; j <= gmax is target row j,
 // j > gmax is draft row j-gmax-1.  Rows a sequence does not have this step are skipped.
 // ---------------------------------------------------------------------------------------------
+template <bool BF16>       // logits stored as bf16 bit patterns (widened exactly) instead of float32
 __global__ void __launch_bounds__(RS_THREADS)
 accept_rowstats_kernel(const __grid_constant__ AcceptLaunch a)
 {
@@ -193,14 +195,14 @@ accept_rowstats_kernel(const __grid_constant__ AcceptLaunch a)
         const int g = seq_gamma(p, b);
         const float T = seq_temperature(p, b);
         const bool greedy = !(T > 0.f);
-        const float *row;
+        const void *row;
         if (j <= p.gamma_max) {
             if (j > g) continue;
-            row = p.target_logits + (long long)(p.cu_q[b] + j) * p.row_stride;
+            row = logit_row<BF16>(p.target_logits, p.cu_q[b] + j, p.row_stride);
         } else {
             const int i = j - p.gamma_max - 1;
             if (i >= g || greedy) continue;
-            row = p.draft_logits + (long long)(p.cu_d[b] + i) * p.row_stride;
+            row = logit_row<BF16>(p.draft_logits, p.cu_d[b] + i, p.row_stride);
         }
         const int lo = slice_id * a.slice;
         const int hi = min(p.vocab, lo + a.slice);
@@ -247,41 +249,7 @@ accept_rowstats_kernel(const __grid_constant__ AcceptLaunch a)
             }
         };
 
-        if (a.vec_ok) {
-            // lo is a multiple of 4; the row base is 16-byte aligned
-            const int n4 = (hi - lo) >> 2;
-            const float *base = row + lo;
-            for (int v0 = lane; v0 < n4; v0 += 32 * RS_UNROLL) {
-                float4 x[RS_UNROLL];
-#pragma unroll
-                for (int u = 0; u < RS_UNROLL; ++u) {
-                    const int v = v0 + u * 32;
-                    x[u] = (v < n4) ? ld_stream_f4(base + 4 * (long long)v)
-                                    : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F,
-                                                  -CUDART_INF_F);
-                }
-#pragma unroll
-                for (int u = 0; u < RS_UNROLL; ++u) {
-                    const int v = v0 + u * 32;
-                    if (v < n4) consume4(x[u].x, x[u].y, x[u].z, x[u].w, lo + 4 * v);
-                }
-            }
-            // ragged tail (vocab not a multiple of 4): at most 3 elements, last slice only
-            const int tail0 = lo + 4 * n4;
-            if (lane == 0 && tail0 < hi) {
-                float t[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) t[u] = (tail0 + u < hi) ? row[tail0 + u] : -CUDART_INF_F;
-                consume4(t[0], t[1], t[2], t[3], tail0);
-            }
-        } else {
-            for (int k0 = lo + 4 * lane; k0 < hi; k0 += 4 * 32) {
-                float t[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) t[u] = (k0 + u < hi) ? __ldg(row + k0 + u) : -CUDART_INF_F;
-                consume4(t[0], t[1], t[2], t[3], k0);
-            }
-        }
+        stream_slice<BF16, RS_UNROLL>(row, lo, hi, a.vec_ok != 0, lane, consume4);
 
         // warp reduction
         if (greedy) {
@@ -333,6 +301,7 @@ __device__ __forceinline__ RowPartial load_partial(const RowPartial *q)
 // ---------------------------------------------------------------------------------------------
 constexpr int DEC_THREADS = 128;
 
+template <bool BF16>
 __device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideScratch *sc, int tid, SeqRecord *rec_out)
 {
     constexpr bool write = true;
@@ -345,8 +314,8 @@ __device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideS
     const bool greedy = !(Tf > 0.f);
     const double T = (double)Tf;
     const int V = p.vocab;
-    const float *t_rows = p.target_logits + (long long)p.cu_q[b] * p.row_stride;
-    const float *d_rows = greedy ? nullptr : p.draft_logits + (long long)p.cu_d[b] * p.row_stride;
+    const void *t_rows = logit_row<BF16>(p.target_logits, p.cu_q[b], p.row_stride);
+    const void *d_rows = greedy ? nullptr : logit_row<BF16>(p.draft_logits, p.cu_d[b], p.row_stride);
     const int32_t *x = p.draft_tokens + p.cu_d[b];
     int32_t *out = p.out_tokens + (long long)b * (gmax + 1);
 
@@ -417,8 +386,8 @@ __device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideS
             if (!(isfinite(lzp) && isfinite(lzq))) {
                 code = 2;
             } else {
-                const double lp = (double)t_rows[(long long)i * p.row_stride + xi] / T - lzp;
-                const double lq = (double)d_rows[(long long)i * p.row_stride + xi] / T - lzq;
+                const double lp = (double)logit_at<BF16>(t_rows, (long long)i * p.row_stride + xi) / T - lzp;
+                const double lq = (double)logit_at<BF16>(d_rows, (long long)i * p.row_stride + xi) / T - lzq;
                 // ratio = min(1, p/q); q == 0 (a token the draft could not have produced) -> 1
                 r = (lq == -CUDART_INF) ? 1.0 : exp(fmin(lp - lq, 0.0));
                 const double u = (double)p.u_accept[p.cu_d[b] + i];
@@ -472,25 +441,14 @@ __device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideS
 
 // Kernel 2: one block per sequence takes the decision; it also clears the sequence's completion
 // counter for kernel 3.
+template <bool BF16>
 __global__ void __launch_bounds__(DEC_THREADS)
 accept_decide_kernel(const __grid_constant__ AcceptLaunch a)
 {
     __shared__ DecideScratch s_dec;
     const int b = blockIdx.x;
     if (threadIdx.x == 0) a.done[b] = 0u;
-    decide_seq(a, b, &s_dec, threadIdx.x, a.records + b);
-}
-
-// four consecutive logits starting at k0 (k0 % 4 == 0), -inf past the vocabulary
-__device__ __forceinline__ void load4(const float *row, int k0, int V, bool vec, float x[4])
-{
-    if (vec && k0 + 3 < V) {
-        const float4 v = *reinterpret_cast<const float4 *>(row + k0);
-        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
-    } else {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) x[u] = (k0 + u < V) ? row[k0 + u] : -CUDART_INF_F;
-    }
+    decide_seq<BF16>(a, b, &s_dec, threadIdx.x, a.records + b);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -502,6 +460,7 @@ __device__ __forceinline__ void load4(const float *row, int k0, int V, bool vec,
 // ---------------------------------------------------------------------------------------------
 constexpr int PICK_SEGS = 2048;     // 2 x 16 KB of shared memory: vocabularies up to 262144
 
+template <bool BF16>
 __device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const SeqRecord &rec, int tid, const double *tab,
                                          double (*s_w)[PICK_SEGS])
 {
@@ -510,8 +469,8 @@ __device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const Seq
     const bool residual = rec.mode == 1;
     const int V = p.vocab, n_seg = a.n_seg, n = rec.n;
     const double c = 1.4426950408889634 / (double)seq_temperature(p, b);
-    const float *trow = p.target_logits + ((long long)p.cu_q[b] + n) * p.row_stride;
-    const float *drow = residual ? p.draft_logits + ((long long)p.cu_d[b] + n) * p.row_stride : nullptr;
+    const void *trow = logit_row<BF16>(p.target_logits, p.cu_q[b] + n, p.row_stride);
+    const void *drow = residual ? logit_row<BF16>(p.draft_logits, p.cu_d[b] + n, p.row_stride) : nullptr;
     const bool vec = a.vec_ok != 0;
     const double ref_p = (double)rec.ref_p, ref_q = (double)rec.ref_q;
     const double *seg_ap = a.seg + (size_t)b * 3 * n_seg, *seg_bp = seg_ap + n_seg, *seg_a = seg_bp + n_seg;
@@ -577,8 +536,8 @@ __device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const Seq
     // exact float64 weights of four consecutive tokens
     auto weights4 = [&](int k0, double w[4]) {
         float xt[4], xd[4];
-        load4(trow, k0, V, vec, xt);
-        if (use_resid) load4(drow, k0, V, vec, xd);
+        logit_load4<BF16>(trow, k0, V, vec, xt);
+        if (use_resid) logit_load4<BF16>(drow, k0, V, vec, xd);
         double y[8], e[8];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -653,6 +612,7 @@ __device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const Seq
 // ---------------------------------------------------------------------------------------------
 // Four blocks (32 warps) per SM: the pass is a mix of float64 arithmetic and shuffles that no
 // pipe saturates, so throughput follows the number of resident warps; 64 registers suffice.
+template <bool BF16>
 __global__ void __launch_bounds__(SEG_THREADS, 4)
 accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
 {
@@ -670,8 +630,8 @@ accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
     const bool residual = rec.mode == 1;
     const int V = p.vocab, n_seg = a.n_seg;
     const double c = 1.4426950408889634 / (double)seq_temperature(p, b);
-    const float *trow = p.target_logits + ((long long)p.cu_q[b] + rec.n) * p.row_stride;
-    const float *drow = residual ? p.draft_logits + ((long long)p.cu_d[b] + rec.n) * p.row_stride : nullptr;
+    const void *trow = logit_row<BF16>(p.target_logits, p.cu_q[b] + rec.n, p.row_stride);
+    const void *drow = residual ? logit_row<BF16>(p.draft_logits, p.cu_d[b] + rec.n, p.row_stride) : nullptr;
     const bool vec = a.vec_ok != 0;
     const double ref_p = (double)rec.ref_p, ref_q = (double)rec.ref_q;
     // first-pass partition sums, good to ~1e-7: only used to decide the sign of p_k - q_k
@@ -689,8 +649,8 @@ accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
         for (int q = 0; q < UN; ++q) {
             const int s = s0 + q * NW;
             if (s < s_end) {
-                load4(trow, s * SEG + 4 * lane, V, vec, xt[q]);
-                if (residual) load4(drow, s * SEG + 4 * lane, V, vec, xd[q]);
+                logit_load4<BF16>(trow, s * SEG + 4 * lane, V, vec, xt[q]);
+                if (residual) logit_load4<BF16>(drow, s * SEG + 4 * lane, V, vec, xd[q]);
             }
         }
 #pragma unroll
@@ -759,7 +719,7 @@ accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
     __syncthreads();
     if (s_last) {             // the same for the whole block
         __threadfence();
-        pick_seq(a, b, rec, tid, s_tab, s_w);
+        pick_seq<BF16>(a, b, rec, tid, s_tab, s_w);
     }
 }
 
@@ -812,6 +772,19 @@ static sv_status check_accept(const sv_accept_params *p)
     return SV_OK;
 }
 
+template <bool BF16>
+static sv_status launch_kernels(const AcceptLaunch &a, int rs_grid, cudaStream_t stream)
+{
+    accept_rowstats_kernel<BF16><<<rs_grid, RS_THREADS, 0, stream>>>(a);
+    sv_status st = launch_check();
+    if (st != SV_OK) return st;
+    accept_decide_kernel<BF16><<<a.p.batch, DEC_THREADS, 0, stream>>>(a);
+    st = launch_check();
+    if (st != SV_OK) return st;
+    accept_sample_kernel<BF16><<<(unsigned)(a.splits * a.p.batch), SEG_THREADS, 0, stream>>>(a);
+    return launch_check();
+}
+
 // the three launches; `scratch` holds accept_layout(..., slice).total bytes
 static sv_status launch_accept(const sv_accept_params *p, void *scratch, int slice, cudaStream_t stream)
 {
@@ -827,8 +800,8 @@ static sv_status launch_accept(const sv_accept_params *p, void *scratch, int sli
     a.slice = slice;
     a.n_slices = (p->vocab + slice - 1) / slice;
     a.n_seg = (p->vocab + SEG - 1) / SEG;
-    a.vec_ok = (p->row_stride % 4 == 0) && aligned16(p->target_logits) &&
-               (p->draft_logits == nullptr || aligned16(p->draft_logits));
+    const bool bf16 = p->logits_bf16 != 0;
+    a.vec_ok = logits_vec_ok(p->target_logits, p->row_stride, bf16) && logits_vec_ok(p->draft_logits, p->row_stride, bf16);
     // blocks per sequence in the sampling kernel: the float64 pass is bound by arithmetic, so
     // several small blocks per SM balance better than one wave of large ones -- two full waves
     // of the four blocks an SM holds (4, 10, 13, 16 blocks per sequence measured slower than 9
@@ -842,25 +815,19 @@ static sv_status launch_accept(const sv_accept_params *p, void *scratch, int sli
 
     const long long n_items = (long long)p->batch * (2 * p->gamma_max + 1) * a.n_slices;
     const long long blocks_needed = (n_items + RS_THREADS / 32 - 1) / (RS_THREADS / 32);
-    static int blocks_per_sm_of[MAX_DEVICES];      // resident blocks per SM, asked once per device
+    static int blocks_per_sm_of[MAX_DEVICES][2];   // resident blocks per SM, asked once per device and logit type
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return SV_ECUDA;
-    if (blocks_per_sm_of[dev] == 0) {
+    if (blocks_per_sm_of[dev][bf16] == 0) {
         int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, accept_rowstats_kernel, RS_THREADS, 0) !=
-                cudaSuccess || n < 1)
-            n = 2;
-        blocks_per_sm_of[dev] = n;
+        const cudaError_t e = bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, accept_rowstats_kernel<true>, RS_THREADS, 0)
+                                   : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, accept_rowstats_kernel<false>, RS_THREADS, 0);
+        if (e != cudaSuccess || n < 1) n = 2;
+        blocks_per_sm_of[dev][bf16] = n;
     }
-    const long long cap = (long long)blocks_per_sm_of[dev] * sm_count();
-    accept_rowstats_kernel<<<(int)(blocks_needed < cap ? blocks_needed : cap), RS_THREADS, 0, stream>>>(a);
-    sv_status st = launch_check();
-    if (st != SV_OK) return st;
-    accept_decide_kernel<<<p->batch, DEC_THREADS, 0, stream>>>(a);
-    st = launch_check();
-    if (st != SV_OK) return st;
-    accept_sample_kernel<<<(unsigned)(splits * p->batch), SEG_THREADS, 0, stream>>>(a);
-    return launch_check();
+    const long long cap = (long long)blocks_per_sm_of[dev][bf16] * sm_count();
+    const int rs_grid = (int)(blocks_needed < cap ? blocks_needed : cap);
+    return bf16 ? launch_kernels<true>(a, rs_grid, stream) : launch_kernels<false>(a, rs_grid, stream);
 }
 
 }  // namespace sv

@@ -222,7 +222,7 @@ extern "C" sv_status spec_verify_step_host(const sv_step_host_io *io, const sv_a
     if (st != SV_OK) return st;
     cudaStream_t s = (cudaStream_t)stream;
     const size_t q_bytes = (size_t)io->n_q_rows * attn->hq * attn->head_dim * 2;
-    const size_t row_bytes = (size_t)acc->row_stride * sizeof(float);
+    const size_t row_bytes = (size_t)acc->row_stride * (acc->logits_bf16 != 0 ? 2 : sizeof(float));
     bool ok = true;
     auto h2d = [&](const void *dst, const void *src, size_t n) {
         if (n != 0 && src != nullptr && dst != nullptr)

@@ -11,6 +11,7 @@
 //     with its lanes over the slice records: merges them, evaluates the confidence c_i = 2^(max * log2(e)/T - ref) / sum in float64 and
 //     takes the first position below tau.
 #include "common.cuh"
+#include "row_stream.cuh"
 
 namespace sv {
 
@@ -49,6 +50,7 @@ __device__ __forceinline__ int ds_gamma(const sv_draft_stop_params &p, int b)
     return g;
 }
 
+template <bool BF16>       // logits stored as bf16 bit patterns (widened exactly) instead of float32
 __global__ void __launch_bounds__(DS_THREADS)
 draft_conf_rowstats_kernel(const __grid_constant__ DraftStopLaunch a)
 {
@@ -64,7 +66,7 @@ draft_conf_rowstats_kernel(const __grid_constant__ DraftStopLaunch a)
         const int b = dense_row / p.gamma_max, i = dense_row % p.gamma_max;
         const float T = ds_temperature(p, b);
         if (i >= ds_gamma(p, b) || !(T > 0.f)) continue;       // no such position, or a greedy draft
-        const float *row = p.draft_logits + (long long)(p.cu_d[b] + i) * p.row_stride;
+        const void *row = logit_row<BF16>(p.draft_logits, p.cu_d[b] + i, p.row_stride);
         const int lo = slice_id * a.slice;
         const int hi = min(p.vocab, lo + a.slice);
 
@@ -79,7 +81,7 @@ draft_conf_rowstats_kernel(const __grid_constant__ DraftStopLaunch a)
         }
         float ref = REF_INIT, amax = -CUDART_INF_F;
         double sum = 0.0;
-        auto consume4 = [&](float x0, float x1, float x2, float x3) {
+        auto consume4 = [&](float x0, float x1, float x2, float x3, int) {
             const float m4 = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
             amax = fmaxf(amax, m4);
             const float ymax = m4 * c_hi + 1.f;
@@ -94,36 +96,7 @@ draft_conf_rowstats_kernel(const __grid_constant__ DraftStopLaunch a)
             const float e3 = ex2_approx(fmaf(x3, c_lo, fmaf(x3, c_hi, -ref)));
             sum += (double)((e0 + e1) + (e2 + e3));
         };
-        if (a.vec_ok) {
-            const int n4 = (hi - lo) >> 2;
-            const float *base = row + lo;
-            for (int v0 = lane; v0 < n4; v0 += 32 * DS_UNROLL) {
-                float4 x[DS_UNROLL];
-#pragma unroll
-                for (int u = 0; u < DS_UNROLL; ++u) {
-                    const int v = v0 + u * 32;
-                    x[u] = (v < n4) ? ld_stream_f4(base + 4 * (long long)v)
-                                    : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
-                }
-#pragma unroll
-                for (int u = 0; u < DS_UNROLL; ++u)
-                    if (v0 + u * 32 < n4) consume4(x[u].x, x[u].y, x[u].z, x[u].w);
-            }
-            const int tail0 = lo + 4 * n4;       // vocab not a multiple of 4: at most 3 elements, last slice only
-            if (lane == 0 && tail0 < hi) {
-                float t[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) t[u] = (tail0 + u < hi) ? row[tail0 + u] : -CUDART_INF_F;
-                consume4(t[0], t[1], t[2], t[3]);
-            }
-        } else {
-            for (int k0 = lo + 4 * lane; k0 < hi; k0 += 4 * 32) {
-                float t[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) t[u] = (k0 + u < hi) ? __ldg(row + k0 + u) : -CUDART_INF_F;
-                consume4(t[0], t[1], t[2], t[3]);
-            }
-        }
+        stream_slice<BF16, DS_UNROLL>(row, lo, hi, a.vec_ok != 0, lane, consume4);
         float r = ref;
 #pragma unroll
         for (int m = 16; m > 0; m >>= 1) {
@@ -237,23 +210,27 @@ extern "C" sv_status spec_draft_stop(const sv_draft_stop_params *p, void *worksp
     a.partials = static_cast<sv::ConfPartial *>(workspace);
     a.slice = sv::ds_pick_slice(p);
     a.n_slices = (p->vocab + a.slice - 1) / a.slice;
-    a.vec_ok = (p->row_stride % 4 == 0) && sv::aligned16(p->draft_logits);
+    const bool bf16 = p->logits_bf16 != 0;
+    a.vec_ok = sv::logits_vec_ok(p->draft_logits, p->row_stride, bf16);
     const long long n_items = (long long)p->batch * p->gamma_max * a.n_slices;
     if (n_items > 0) {
-        static int blocks_per_sm_of[64];    // resident blocks per SM, asked once per device
+        static int blocks_per_sm_of[64][2]; // resident blocks per SM, asked once per device and logit type
         int dev = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SV_ECUDA;
-        if (blocks_per_sm_of[dev] == 0) {
+        if (blocks_per_sm_of[dev][bf16] == 0) {
             int n = 0;
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, sv::draft_conf_rowstats_kernel, sv::DS_THREADS,
-                                                              0) != cudaSuccess || n < 1)
-                n = 2;
-            blocks_per_sm_of[dev] = n;
+            const cudaError_t e =
+                bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, sv::draft_conf_rowstats_kernel<true>, sv::DS_THREADS, 0)
+                     : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, sv::draft_conf_rowstats_kernel<false>, sv::DS_THREADS, 0);
+            if (e != cudaSuccess || n < 1) n = 2;
+            blocks_per_sm_of[dev][bf16] = n;
         }
-        const int blocks_per_sm = blocks_per_sm_of[dev];
+        const int blocks_per_sm = blocks_per_sm_of[dev][bf16];
         const long long blocks_needed = (n_items + sv::DS_THREADS / 32 - 1) / (sv::DS_THREADS / 32);
         const long long cap = (long long)blocks_per_sm * sv::sm_count();
-        sv::draft_conf_rowstats_kernel<<<(int)(blocks_needed < cap ? blocks_needed : cap), sv::DS_THREADS, 0, s>>>(a);
+        const int grid = (int)(blocks_needed < cap ? blocks_needed : cap);
+        if (bf16) sv::draft_conf_rowstats_kernel<true><<<grid, sv::DS_THREADS, 0, s>>>(a);
+        else sv::draft_conf_rowstats_kernel<false><<<grid, sv::DS_THREADS, 0, s>>>(a);
         const sv_status st = sv::launch_check();
         if (st != SV_OK) return st;
     }

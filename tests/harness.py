@@ -129,13 +129,21 @@ class AcceptOut:
     status: int
 
 
+def bf16_rounded(li: synth.LogitInputs) -> synth.LogitInputs:
+    """The same inputs with every logit rounded to bf16 (held as float32: the oracle's view of bf16 logits)."""
+    r = lambda x: synth.bf16_to_f32(synth.bf16_bits(x)).reshape(x.shape)
+    return synth.LogitInputs(r(li.target_logits), r(li.draft_logits), li.draft_tokens, li.u_accept, li.u_sample)
+
+
 def run_accept_gpu(li: synth.LogitInputs, temperature, gamma, cu_q, cu_d, gamma_max,
-                   temperature_per_seq=None) -> AcceptOut:
+                   temperature_per_seq=None, bf16=False) -> AcceptOut:
+    """bf16: the logits (already bf16-representable, see bf16_rounded) go to the device as bf16 tensors."""
     B = len(gamma)
     V = li.target_logits.shape[1]
     n_q, n_d = int(cu_q[-1]), int(cu_d[-1])
-    tl = dev(li.target_logits)
-    dl = dev(li.draft_logits) if n_d > 0 else torch.zeros((1, V), dtype=torch.float32, device=DEV)
+    ldt = torch.bfloat16 if bf16 else torch.float32
+    tl = dev(li.target_logits).to(ldt)
+    dl = dev(li.draft_logits).to(ldt) if n_d > 0 else torch.zeros((1, V), dtype=ldt, device=DEV)
     x = dev(li.draft_tokens) if n_d > 0 else torch.zeros(1, dtype=torch.int32, device=DEV)
     ua = dev(li.u_accept) if n_d > 0 else torch.zeros(1, dtype=torch.float32, device=DEV)
     us = dev(li.u_sample)
@@ -197,9 +205,9 @@ def compare_accept(gpu: AcceptOut, li: synth.LogitInputs, temperature, gamma, cu
     return ref, n_flag_pos, n_flag_tok
 
 
-def check_accept(li, temperature, gamma, cu_q, cu_d, gamma_max, temperature_per_seq=None):
+def check_accept(li, temperature, gamma, cu_q, cu_d, gamma_max, temperature_per_seq=None, bf16=False):
     T = temperature_per_seq if temperature_per_seq is not None else temperature
-    gpu = run_accept_gpu(li, temperature, gamma, cu_q, cu_d, gamma_max, temperature_per_seq)
+    gpu = run_accept_gpu(li, temperature, gamma, cu_q, cu_d, gamma_max, temperature_per_seq, bf16)
     assert gpu.status == 0, f"device status {gpu.status}"
     ref, n_pos, n_tok = compare_accept(gpu, li, T, gamma, cu_q, cu_d, gamma_max)
     # softmax sums (fp32 exponentials): Z relative error <= 1e-5, i.e. |d lnZ| <= 1e-5

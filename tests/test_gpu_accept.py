@@ -228,6 +228,28 @@ def test_device_status_bits():
         np.testing.assert_array_equal(gpu.out_tokens[b], ref.out_tokens[b])
 
 
+@pytest.mark.parametrize("name", ["c1", "c3", "c4"])
+def test_bf16_logits(name):
+    """Logits stored as bf16: the device widens them exactly, so the result is the oracle's on the widened values
+    (the same bit-exact comparison as for float32 logits), for the vectorised and the element-wise loads."""
+    from tests.harness import bf16_rounded
+    cfg = synth.CONFIGS[name]
+    if name == "c4":
+        cfg = synth.scaled(cfg, batch=8)
+    li, g, cu_q, cu_d = case(cfg, padded=(name == "c4"))
+    check_accept(bf16_rounded(li), cfg.temperature, g, cu_q, cu_d, cfg.gamma_max, bf16=True)
+    check_accept(bf16_rounded(synth.LogitInputs(li.target_logits, li.draft_logits, li.draft_tokens, li.u_accept,
+                                                li.u_sample)), 0.0, g, cu_q, cu_d, cfg.gamma_max, bf16=True)
+
+
+@pytest.mark.parametrize("V", [1, 5, 8, 1000, 4099])
+def test_bf16_logits_small_and_odd_vocabularies(V):
+    from tests.harness import bf16_rounded
+    cfg = synth.VerifyConfig("odd16", 3, 1, 1, 64, V, 32, 32, 0, 3, 3, 0.9, 0.7, seed=91 + V)
+    li, g, cu_q, cu_d = case(cfg)
+    check_accept(bf16_rounded(li), cfg.temperature, g, cu_q, cu_d, cfg.gamma_max, bf16=True)
+
+
 def test_greedy_rows_without_an_argmax_set_the_status_bit():
     """T = 0: a target row that is all -inf, or holds a NaN or +inf, has no argmax.  The header promises
     SV_DEV_NONFINITE, no accepted drafts and -1 tokens for such a sequence, and nothing else changes."""

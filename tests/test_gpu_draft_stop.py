@@ -13,11 +13,12 @@ from tests.harness import DEV, dev, workspace
 pytestmark = pytest.mark.gpu
 
 
-def run_gpu(draft_logits, T, tau, gamma, cu_d, gamma_max, T_per_seq=None):
+def run_gpu(draft_logits, T, tau, gamma, cu_d, gamma_max, T_per_seq=None, bf16=False):
     B = len(gamma)
     n_d = int(cu_d[-1])
     V = draft_logits.shape[1]
-    dl = dev(draft_logits) if n_d > 0 else torch.zeros((1, V), dtype=torch.float32, device=DEV)
+    ldt = torch.bfloat16 if bf16 else torch.float32      # bf16: the values are bf16-representable already
+    dl = dev(draft_logits).to(ldt) if n_d > 0 else torch.zeros((1, V), dtype=ldt, device=DEV)
     n = torch.full((B,), -7, dtype=torch.int32, device=DEV)
     top = torch.full((max(n_d, 1),), float("nan"), dtype=torch.float64, device=DEV)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
@@ -29,9 +30,9 @@ def run_gpu(draft_logits, T, tau, gamma, cu_d, gamma_max, T_per_seq=None):
     return n.cpu().numpy(), top.cpu().numpy()[:n_d], int(status.item())
 
 
-def check(draft_logits, T, tau, gamma, cu_d, gamma_max, T_per_seq=None):
+def check(draft_logits, T, tau, gamma, cu_d, gamma_max, T_per_seq=None, bf16=False):
     Tref = T_per_seq if T_per_seq is not None else T
-    n_gpu, top_gpu, status = run_gpu(draft_logits, T, tau, gamma, cu_d, gamma_max, T_per_seq)
+    n_gpu, top_gpu, status = run_gpu(draft_logits, T, tau, gamma, cu_d, gamma_max, T_per_seq, bf16)
     assert status == 0
     n_ref, top_ref, flag = oracle.draft_stop(draft_logits, Tref, tau, gamma, cu_d)
     if len(top_ref):
@@ -82,6 +83,18 @@ def test_small_and_odd_vocabularies(V):
     d = (rng.standard_normal((int(cu_d[-1]), V)) * 2.0).astype(np.float32)
     _, top, _ = oracle.draft_stop(d, 1.0, 0.0, gamma, cu_d)
     check(d, 1.0, float(np.median(top)), gamma, cu_d, 5)
+
+
+@pytest.mark.parametrize("V", [3, 8, 1001, 32000])
+def test_bf16_logits(V):
+    # draft rows stored as bf16: widened exactly on the device, so the oracle sees the same values
+    rng = np.random.default_rng(100 + V)
+    gamma = np.array([3, 0, 5, 1, 4], np.int32)
+    cu_d = np.concatenate([[0], np.cumsum(gamma)]).astype(np.int32)
+    d = (rng.standard_normal((int(cu_d[-1]), V)) * 2.0).astype(np.float32)
+    d = synth.bf16_to_f32(synth.bf16_bits(d)).reshape(d.shape)
+    _, top, _ = oracle.draft_stop(d, 1.0, 0.0, gamma, cu_d)
+    check(d, 1.0, float(np.median(top)), gamma, cu_d, 5, bf16=True)
 
 
 def test_longest_draft_blocks():
