@@ -571,7 +571,7 @@ def run_ours(args):
         cfg, seq_len, gamma, cu_q, cu_d = workload_inputs(base_cfg, rank, args.batch, args.gamma, args.gamma_max)
     if world == 1 and not args.no_cpu_baseline:
         import oracle
-        n_seq = min(args.oracle_seqs or 16, B)
+        n_seq = min(args.oracle_seqs or 64, B)
         sub, kv_s, q_s, li_s = sample_inputs(cfg, seq_len, gamma, cu_q, cu_d, n_seq)
         dt, otoks = oracle_step(sub, seq_len, gamma, cu_q, cu_d, kv_s, q_s, li_s, n_seq)
         line["cpu_baseline"] = {"value": otoks / dt, "unit": UNIT, "cores": oracle.num_threads(),

@@ -241,11 +241,24 @@ accept_rowstats_kernel(const __grid_constant__ AcceptLaunch a)
                     sum = scale_down_pow2(sum, ref - nr);
                     ref = nr;
                 }
-                const float e0 = ex2_approx(fmaf(x0, c_lo, fmaf(x0, c_hi, -ref)));
-                const float e1 = ex2_approx(fmaf(x1, c_lo, fmaf(x1, c_hi, -ref)));
-                const float e2 = ex2_approx(fmaf(x2, c_lo, fmaf(x2, c_hi, -ref)));
-                const float e3 = ex2_approx(fmaf(x3, c_lo, fmaf(x3, c_hi, -ref)));
-                sum += (double)((e0 + e1) + (e2 + e3));
+                if (BF16) {
+                    // With bf16 logits the pass is bound by instruction issue, not by memory: two logits
+                    // per instruction (packed float32 pairs; each half rounds as the scalar form does).
+                    // With float32 logits the scalar form measured slightly faster.
+                    const float2 ch2 = make_float2(c_hi, c_hi), cl2 = make_float2(c_lo, c_lo), nr2 = make_float2(-ref, -ref);
+                    const float2 xa = make_float2(x0, x2), xb = make_float2(x1, x3);
+                    const float2 ya = __ffma2_rn(xa, cl2, __ffma2_rn(xa, ch2, nr2));
+                    const float2 yb = __ffma2_rn(xb, cl2, __ffma2_rn(xb, ch2, nr2));
+                    const float2 e = __fadd2_rn(make_float2(ex2_approx(ya.x), ex2_approx(ya.y)),
+                                                make_float2(ex2_approx(yb.x), ex2_approx(yb.y)));    // (e0 + e1, e2 + e3)
+                    sum += (double)(e.x + e.y);
+                } else {
+                    const float e0 = ex2_approx(fmaf(x0, c_lo, fmaf(x0, c_hi, -ref)));
+                    const float e1 = ex2_approx(fmaf(x1, c_lo, fmaf(x1, c_hi, -ref)));
+                    const float e2 = ex2_approx(fmaf(x2, c_lo, fmaf(x2, c_hi, -ref)));
+                    const float e3 = ex2_approx(fmaf(x3, c_lo, fmaf(x3, c_hi, -ref)));
+                    sum += (double)((e0 + e1) + (e2 + e3));
+                }
             }
         };
 
