@@ -304,23 +304,36 @@ class VerifyStep:
         self.seq_len = self.sl.cpu().numpy().copy()
 
     def timed(self, steps, warmup, barrier):
+        """Whole-step time from one pair of events around `steps` steps enqueued back to back (nothing but the
+        step's own calls and the state reset on the stream, so that each kernel can be set up while its
+        predecessor drains), then the same number of steps again with an event after every call for the
+        breakdown."""
         torch = self.torch
         for _ in range(warmup):
             self.step()
         barrier()
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
         e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         launches0 = self.sv.sv_launch_count()
         barrier()
         e_begin.record(self.stream)
         for it in range(steps):
-            self.step(evs[it])
+            self.step()
         e_end.record(self.stream)
         barrier()
+        launches = self.sv.sv_launch_count() - launches0
         assert self.status.item() == 0, f"device status {self.status.item()}"
-        return {"ms_total": e_begin.elapsed_time(e_end),
-                "tokens": int((self.n_acc + 1).sum().item()),           # identical every step (same inputs, same state)
-                "launches": self.sv.sv_launch_count() - launches0,
+        tokens = int((self.n_acc + 1).sum().item())           # identical every step (same inputs, same state)
+        # The breakdown pass: after a pause and a short warm-up, so that it runs in the clock state of the timed
+        # pass (this GPU lowers its SM clock after about 50 ms of continuous load; the timed pass ends before that).
+        time.sleep(0.5)
+        for _ in range(3):
+            self.step()
+        barrier()
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+        for it in range(steps):
+            self.step(evs[it])
+        barrier()
+        return {"ms_total": e_begin.elapsed_time(e_end), "tokens": tokens, "launches": launches,
                 "attn": float(np.mean([e[0].elapsed_time(e[1]) for e in evs])),
                 "accept": float(np.mean([e[1].elapsed_time(e[2]) for e in evs])),
                 "gamma": float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))}

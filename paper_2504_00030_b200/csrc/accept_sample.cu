@@ -180,6 +180,7 @@ template <bool BF16>       // logits stored as bf16 bit patterns (widened exactl
 __global__ void __launch_bounds__(RS_THREADS)
 accept_rowstats_kernel(const __grid_constant__ AcceptLaunch a)
 {
+    pdl_enter();
     const sv_accept_params &p = a.p;
     const int rows_per_seq = 2 * p.gamma_max + 1;
     const long long n_items = (long long)p.batch * rows_per_seq * a.n_slices;
@@ -458,6 +459,7 @@ template <bool BF16>
 __global__ void __launch_bounds__(DEC_THREADS)
 accept_decide_kernel(const __grid_constant__ AcceptLaunch a)
 {
+    pdl_enter();
     __shared__ DecideScratch s_dec;
     const int b = blockIdx.x;
     if (threadIdx.x == 0) a.done[b] = 0u;
@@ -629,6 +631,7 @@ template <bool BF16>
 __global__ void __launch_bounds__(SEG_THREADS, 4)
 accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
 {
+    pdl_enter();
     const sv_accept_params &p = a.p;
     __shared__ double s_tab[128];
     __shared__ double s_red[2 * (SEG_THREADS / 32)];
@@ -788,14 +791,11 @@ static sv_status check_accept(const sv_accept_params *p)
 template <bool BF16>
 static sv_status launch_kernels(const AcceptLaunch &a, int rs_grid, cudaStream_t stream)
 {
-    accept_rowstats_kernel<BF16><<<rs_grid, RS_THREADS, 0, stream>>>(a);
-    sv_status st = launch_check();
+    sv_status st = launch_kernel(false, accept_rowstats_kernel<BF16>, rs_grid, RS_THREADS, 0, stream, a);
     if (st != SV_OK) return st;
-    accept_decide_kernel<BF16><<<a.p.batch, DEC_THREADS, 0, stream>>>(a);
-    st = launch_check();
+    st = launch_kernel(true, accept_decide_kernel<BF16>, a.p.batch, DEC_THREADS, 0, stream, a);
     if (st != SV_OK) return st;
-    accept_sample_kernel<BF16><<<(unsigned)(a.splits * a.p.batch), SEG_THREADS, 0, stream>>>(a);
-    return launch_check();
+    return launch_kernel(true, accept_sample_kernel<BF16>, (unsigned)(a.splits * a.p.batch), SEG_THREADS, 0, stream, a);
 }
 
 // the three launches; `scratch` holds accept_layout(..., slice).total bytes

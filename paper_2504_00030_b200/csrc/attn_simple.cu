@@ -39,6 +39,7 @@ __device__ __forceinline__ float block_sum(float v, float *red)
 __global__ void __launch_bounds__(AS_THREADS)
 attn_simple_kernel(sv_attn_params p, sv_kv_pool pool)
 {
+    pdl_enter();
     __shared__ float s_q[128];
     __shared__ float s_p[AS_THREADS];
     __shared__ int s_page[AS_THREADS];
@@ -133,8 +134,7 @@ attn_simple_kernel(sv_attn_params p, sv_kv_pool pool)
 sv_status launch_attn_simple(const sv_attn_params &p, cudaStream_t stream)
 {
     dim3 grid((unsigned)(p.batch * (p.gamma_max + 1)), (unsigned)p.hq);
-    attn_simple_kernel<<<grid, AS_THREADS, 0, stream>>>(p, *p.pool);
-    return launch_check();
+    return launch_kernel(true, attn_simple_kernel, grid, AS_THREADS, 0, stream, p, *p.pool);
 }
 
 }  // namespace sv

@@ -64,6 +64,7 @@ attn_tc_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
     constexpr int SLOT_BYTES = TILE * HD * 2;          // one K or one V tile
     constexpr int O_COL0 = 2 * TILE;                   // TMEM: two S buffers of TILE columns, then O
     constexpr uint32_t TMEM_COLS = (2 * TILE + 128 * NQ <= 256) ? 256u : 512u;
+    pdl_enter();
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // carve: [Q groups][ring slots][Shared]; the swizzled tiles need a 1024-byte aligned base
     uint8_t *smem = smem_raw;
@@ -486,6 +487,7 @@ constexpr int COMBINE_LIST = 64;      // partial slots merged per pass
 __global__ void __launch_bounds__(COMBINE_THREADS)
 attn_combine_kernel(const AttnTcLaunch a)
 {
+    pdl_enter();
     const sv_attn_params &p = a.p;
     __shared__ int s_list[COMBINE_LIST];
     __shared__ int s_n;
@@ -659,8 +661,7 @@ static sv_status launch_main(AttnTcLaunch &a, const sv_attn_params &p, int grid,
     if (cudaFuncSetAttribute(attn_tc_kernel<NQ, TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)
         return SV_ECUDA;
-    attn_tc_kernel<NQ, TILE><<<grid, 128 + 128 * NQ, smem, stream>>>(a, p.pool->k_map, p.pool->v_map);
-    return launch_check();
+    return launch_kernel(false, attn_tc_kernel<NQ, TILE>, grid, 128 + 128 * NQ, smem, stream, a, p.pool->k_map, p.pool->v_map);
 }
 
 sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t workspace_bytes,
@@ -684,8 +685,7 @@ sv_status launch_attn_tc(const sv_attn_params &p, void *workspace, size_t worksp
     if (use_tq) st = launch_attn_tq_main(a, p, grid, stream);
     else st = launch_main<2, 128>(a, p, grid, stream);
     if (st != SV_OK) return st;
-    attn_combine_kernel<<<grid, COMBINE_THREADS, 0, stream>>>(a);
-    return launch_check();
+    return launch_kernel(true, attn_combine_kernel, grid, COMBINE_THREADS, 0, stream, a);
 }
 
 }  // namespace sv

@@ -109,6 +109,7 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
 {
     constexpr bool TAIL = NB > 0;
     constexpr int NBA = NB > 0 ? NB : 1;               // array extent (no zero-length arrays)
+    pdl_enter();
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // carve: [ring slots][tail merge buffers][Shared]; the swizzled tiles need a 1024-byte aligned base
     uint8_t *ring = smem_raw;
@@ -801,8 +802,7 @@ static sv_status launch_tq(AttnTcLaunch &a, const sv_attn_params &p, int grid, c
     if (cudaFuncSetAttribute(attn_tq_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
         return SV_ECUDA;
-    attn_tq_kernel<NB><<<grid, TAIL ? 384 : 256, smem, stream>>>(a, p.pool->k_map, p.pool->v_map);
-    return launch_check();
+    return launch_kernel(false, attn_tq_kernel<NB>, grid, TAIL ? 384 : 256, smem, stream, a, p.pool->k_map, p.pool->v_map);
 }
 
 sv_status launch_attn_tq_main(AttnTcLaunch &a, const sv_attn_params &p, int grid, cudaStream_t stream)

@@ -54,6 +54,7 @@ template <bool BF16>       // logits stored as bf16 bit patterns (widened exactl
 __global__ void __launch_bounds__(DS_THREADS)
 draft_conf_rowstats_kernel(const __grid_constant__ DraftStopLaunch a)
 {
+    pdl_enter();
     const sv_draft_stop_params &p = a.p;
     const long long n_items = (long long)p.batch * p.gamma_max * a.n_slices;
     const int lane = threadIdx.x & 31;
@@ -119,6 +120,7 @@ constexpr int DSD_THREADS = 128;
 __global__ void __launch_bounds__(DSD_THREADS)
 draft_stop_decide_kernel(const __grid_constant__ DraftStopLaunch a)
 {
+    pdl_enter();
     const sv_draft_stop_params &p = a.p;
     __shared__ unsigned char s_below[DS_MAX_GAMMA];
     const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -229,11 +231,9 @@ extern "C" sv_status spec_draft_stop(const sv_draft_stop_params *p, void *worksp
         const long long blocks_needed = (n_items + sv::DS_THREADS / 32 - 1) / (sv::DS_THREADS / 32);
         const long long cap = (long long)blocks_per_sm * sv::sm_count();
         const int grid = (int)(blocks_needed < cap ? blocks_needed : cap);
-        if (bf16) sv::draft_conf_rowstats_kernel<true><<<grid, sv::DS_THREADS, 0, s>>>(a);
-        else sv::draft_conf_rowstats_kernel<false><<<grid, sv::DS_THREADS, 0, s>>>(a);
-        const sv_status st = sv::launch_check();
+        const sv_status st = bf16 ? sv::launch_kernel(false, sv::draft_conf_rowstats_kernel<true>, grid, sv::DS_THREADS, 0, s, a)
+                                  : sv::launch_kernel(false, sv::draft_conf_rowstats_kernel<false>, grid, sv::DS_THREADS, 0, s, a);
         if (st != SV_OK) return st;
     }
-    sv::draft_stop_decide_kernel<<<p->batch, sv::DSD_THREADS, 0, s>>>(a);
-    return sv::launch_check();
+    return sv::launch_kernel(true, sv::draft_stop_decide_kernel, p->batch, sv::DSD_THREADS, 0, s, a);
 }

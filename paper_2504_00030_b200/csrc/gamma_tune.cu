@@ -32,6 +32,7 @@ template <bool INIT>
 __global__ void __launch_bounds__(GT_THREADS)
 gamma_tune_kernel(sv_gamma_params p, int gamma0)
 {
+    pdl_enter();
     __shared__ int scan_smem[16];
     __shared__ int carry[2];
     if (threadIdx.x == 0) {
@@ -137,8 +138,7 @@ extern "C" sv_status gamma_tune_update(const sv_gamma_params *p, void *stream)
 {
     sv_status st = sv::check_params(p, false);
     if (st != SV_OK) return st;
-    sv::gamma_tune_kernel<false><<<1, sv::GT_THREADS, 0, (cudaStream_t)stream>>>(*p, 0);
-    return sv::launch_check();
+    return sv::launch_kernel(true, sv::gamma_tune_kernel<false>, 1, sv::GT_THREADS, 0, (cudaStream_t)stream, *p, 0);
 }
 
 extern "C" sv_status gamma_tune_init(const sv_gamma_params *p, int32_t gamma0, void *stream)
@@ -146,6 +146,5 @@ extern "C" sv_status gamma_tune_init(const sv_gamma_params *p, int32_t gamma0, v
     sv_status st = sv::check_params(p, true);
     if (st != SV_OK) return st;
     if (gamma0 < 0 || gamma0 > p->config.gamma_max) return SV_EINVAL;
-    sv::gamma_tune_kernel<true><<<1, sv::GT_THREADS, 0, (cudaStream_t)stream>>>(*p, gamma0);
-    return sv::launch_check();
+    return sv::launch_kernel(true, sv::gamma_tune_kernel<true>, 1, sv::GT_THREADS, 0, (cudaStream_t)stream, *p, gamma0);
 }

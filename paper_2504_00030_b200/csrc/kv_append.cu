@@ -33,6 +33,7 @@ struct KvAppendLaunch {
 __global__ void __launch_bounds__(KA_THREADS)
 kv_append_kernel(const __grid_constant__ KvAppendLaunch a)
 {
+    pdl_enter();
     const sv_kv_append_params &p = a.p;
     const int rows_max = p.gamma_max + 1;
     const int b = blockIdx.x / rows_max, i = blockIdx.x % rows_max;
@@ -110,8 +111,7 @@ sv_status launch_kv_append_layers(const sv_kv_append_params &shared, const sv_kv
             if (st != SV_OK) return st;
         }
         const dim3 grid((unsigned)(shared.batch * (shared.gamma_max + 1)), (unsigned)n);
-        kv_append_kernel<<<grid, KA_THREADS, 0, stream>>>(a);
-        const sv_status st = launch_check();
+        const sv_status st = launch_kernel(true, kv_append_kernel, grid, KA_THREADS, 0, stream, a);
         if (st != SV_OK) return st;
     }
     return SV_OK;

@@ -12,6 +12,7 @@ namespace sv {
 __global__ void __launch_bounds__(128)
 wait_expiry_kernel(uint32_t *status, int32_t *result, long long limit_cycles)
 {
+    pdl_enter();
     __shared__ uint64_t bar;
     __shared__ int abort_flag;
     if (threadIdx.x == 0) {
@@ -33,6 +34,6 @@ extern "C" sv_status sv_selftest_wait_expiry(uint32_t *device_status, int32_t *d
 {
     if (device_status == nullptr || device_result == nullptr) return SV_EINVAL;
     if (limit_cycles < 1 || limit_cycles > 2000000000LL) return SV_EINVAL;     // at most about a second
-    sv::wait_expiry_kernel<<<1, 128, 0, (cudaStream_t)stream>>>(device_status, device_result, (long long)limit_cycles);
-    return sv::launch_check();
+    return sv::launch_kernel(true, sv::wait_expiry_kernel, 1, 128, 0, (cudaStream_t)stream, device_status, device_result,
+                          (long long)limit_cycles);
 }

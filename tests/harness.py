@@ -87,7 +87,15 @@ def used_rows(gamma, cu_q):
     return np.concatenate([np.arange(cu_q[b], cu_q[b] + gamma[b] + 1) for b in range(len(gamma))])
 
 
-ATTN_ATOL = 2e-2        # bf16 attention outputs, absolute (no allowance for large outputs)
+ATTN_ATOL = 2e-2        # bf16 attention outputs, absolute
+
+
+def attn_allowed(o_ref):
+    """2e-2 absolute.  A bf16 value of magnitude >= 4 is a multiple of 2^-5, so its correctly
+    rounded result can already sit 0.0156 from the exact one; for those elements (reached only
+    by the peaky stress cases) half a bf16 ulp of the reference is added to the bound."""
+    a = np.abs(o_ref)
+    return ATTN_ATOL + np.where(a >= 4.0, a * 2.0 ** -8, 0.0)
 
 
 SUM_RTOL = 1e-5         # fp32 softmax sums, relative
@@ -100,8 +108,8 @@ def check_attn(case: AttnCase):
     assert status == 0, f"device status {status}"
     diff = np.abs(o_gpu[rows] - o_ref[rows])
     err = diff.max()
-    w = np.unravel_index(np.argmax(diff), diff.shape)
-    assert (diff <= ATTN_ATOL).all(), \
+    w = np.unravel_index(np.argmax(diff - attn_allowed(o_ref[rows])), diff.shape)
+    assert (diff <= attn_allowed(o_ref[rows])).all(), \
         f"attention output error {diff[w]} at used-row {w}: gpu {o_gpu[rows][w]} vs oracle {o_ref[rows][w]}"
     # softmax sums: exp(lse) relative error
     rel = np.abs(np.expm1(lse_gpu[rows] - lse_ref[rows])).max()
