@@ -53,7 +53,7 @@ static bool make_pool_map(CUtensorMap *map, const void *base, const sv_kv_pool &
                                 (cuuint64_t)pool.hkv, (cuuint64_t)pool.n_pages};
     const cuuint64_t strides[3] = {(cuuint64_t)pool.strides[2] * 2, (cuuint64_t)pool.strides[1] * 2,
                                    (cuuint64_t)pool.strides[0] * 2};
-    const cuuint32_t box[4] = {64, 16, 1, 1};      // 64 dims (128 B) x 16 slots of one head, one page
+    const cuuint32_t box[4] = {64, 16, 1, 1};      // 64 dims (128 B) x 16 slots of one head, one page (head_dim 128: two boxes per page)
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box,
               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -102,7 +102,7 @@ extern "C" sv_status spec_kv_pool_register(const void *k_pool, const void *v_poo
     pool->head_dim = head_dim;
     for (int i = 0; i < 4; ++i) pool->strides[i] = strides[i];
     pool->has_maps = false;
-    if (head_dim == 128) {
+    if (head_dim == 128 || head_dim == 64) {
         if (!sv::make_pool_map(&pool->k_map, k_pool, *pool) ||
             !sv::make_pool_map(&pool->v_map, v_pool, *pool)) {
             delete pool;

@@ -11,7 +11,7 @@ struct sv_kv_pool {
     int64_t n_pages;
     int32_t page_size, hkv, head_dim;
     int64_t strides[4];     // elements: page, head, slot, dim
-    bool has_maps;          // TMA tensor maps built (head_dim 128 only)
+    bool has_maps;          // TMA tensor maps built (head_dim 128 and 64)
     CUtensorMap k_map;      // 4-D tiled maps over the pool, box = 64 dims x 16 slots of one
     CUtensorMap v_map;      // head of one page, 128-byte swizzle
 };
@@ -22,7 +22,7 @@ namespace sv {
 // used for shapes the tensor-core kernel does not cover and as a tiny-problem path.
 sv_status launch_attn_simple(const sv_attn_params &p, cudaStream_t stream);
 
-// Attention on tcgen05 tensor cores with TMA-staged K/V pages (head_dim 128).
+// Attention on tcgen05 tensor cores with TMA-staged K/V pages (head_dim 128 and 64).
 bool attn_tc_supported(const sv_attn_params &p);
 size_t attn_tc_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t hq, int32_t hkv,
                                int32_t head_dim, int32_t max_seq_len);

@@ -536,6 +536,8 @@ attn_combine_kernel(const AttnTcLaunch a)
     gam = min(max(gam, 0), p.gamma_max);
     const int G = a.group, n_rows = G * (gam + 1);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const int D = p.head_dim;                              // 128, or 64 (rows keep their 128-float pitch in the slots)
+    const bool lane_on = 4 * lane < D;
     const size_t m_off = (size_t)slot_rows * HD, l_off = m_off + (size_t)slot_rows;
     const size_t slot_floats = part_slot_floats(slot_rows);
 
@@ -574,8 +576,8 @@ attn_combine_kernel(const AttnTcLaunch a)
                     const float *slot = a.ws_part + (size_t)s_list[have ? j0 + u : 0] * slot_floats;
                     mc[u] = have ? slot[m_off + r] : -CUDART_INF_F;
                     lc[u] = have ? slot[l_off + r] : 0.f;
-                    v[u] = have ? reinterpret_cast<const float4 *>(slot + (size_t)r * HD)[lane]
-                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                    v[u] = (have && lane_on) ? reinterpret_cast<const float4 *>(slot + (size_t)r * HD)[lane]
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
                 float m_new = m_run;
 #pragma unroll
@@ -595,7 +597,7 @@ attn_combine_kernel(const AttnTcLaunch a)
             }
             if (!last) {
                 float *slot = a.ws_part + (size_t)carry * slot_floats;
-                reinterpret_cast<float4 *>(slot + (size_t)r * HD)[lane] = acc;
+                if (lane_on) reinterpret_cast<float4 *>(slot + (size_t)r * HD)[lane] = acc;
                 if (lane == 0) { slot[m_off + r] = m_run; slot[l_off + r] = l_run; }
                 continue;
             }
@@ -607,7 +609,7 @@ attn_combine_kernel(const AttnTcLaunch a)
             uint2 packed;
             packed.x = *reinterpret_cast<const uint32_t *>(&lo);
             packed.y = *reinterpret_cast<const uint32_t *>(&hi);
-            reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.o) + q_row * HD)[lane] = packed;
+            if (lane_on) reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.o) + q_row * D)[lane] = packed;
             if (lane == 0 && p.lse != nullptr) p.lse[q_row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
         }
     }
@@ -622,10 +624,10 @@ static int rows_groups(const sv_attn_params &p)
 
 bool attn_tc_supported(const sv_attn_params &p)
 {
-    if (p.head_dim != HD || p.pool == nullptr || !p.pool->has_maps) return false;
-    if (p.batch > MAX_BATCH_TC) return false;
+    if (p.pool == nullptr || !p.pool->has_maps || p.batch > MAX_BATCH_TC) return false;
+    if (attn_tq_supported(p)) return true;               // 128 or 64 dims, one row group (+ tail rows)
     const int nq = rows_groups(p);
-    return nq >= 1 && nq <= 2;
+    return p.head_dim == HD && nq >= 1 && nq <= 2;       // two row groups: 128 dims only
 }
 
 static size_t prefix_bytes(int batch)
@@ -640,7 +642,7 @@ size_t attn_tc_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t hq, int
                                int32_t head_dim, int32_t max_seq_len)
 {
     (void)max_seq_len;
-    if (head_dim != HD || hkv <= 0 || hq % hkv != 0) return 0;
+    if ((head_dim != HD && head_dim != 64) || hkv <= 0 || hq % hkv != 0) return 0;
     const int rows = (hq / hkv) * (gamma_max + 1);
     const int nq = (rows + 127) / 128;
     if (nq < 1 || nq > 2 || batch > MAX_BATCH_TC) return 0;

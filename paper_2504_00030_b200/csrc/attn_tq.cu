@@ -31,7 +31,6 @@ namespace sv {
 namespace tq {
 
 constexpr int TILE = 128;                          // tokens per key tile
-constexpr int SLOT_BYTES = TILE * HD * 2;          // one K or one V tile: 32 KB
 constexpr int S_COL0 = 0;                          // TMEM columns: two S buffers,
 constexpr int O_COL0 = 256;                        // the O accumulator,
 constexpr int Q_COL0 = 384;                        // the query rows (bf16 pairs)
@@ -102,12 +101,17 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 
 using namespace tq;
 
-template <int NB>      // blocks of 8 tail rows beyond row 127 (0: no tail warps)
+// NB: blocks of 8 tail rows beyond row 127 (0: no tail warps).  D: head_dim, 128 or 64.  With 64 dims a K or V
+// tile is one 16 KB half (the 128-byte rows of one swizzle atom), Q K^T has four k-steps, O has 64 columns; the
+// partial-result slots keep their 128-float row pitch.
+template <int NB, int D>
 __global__ void __launch_bounds__(NB > 0 ? 384 : 256, 1)
 attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                const __grid_constant__ CUtensorMap v_map)
 {
+    static_assert(D == 128 || (D == 64 && NB == 0), "tail rows are built for 128-dim heads only");
     constexpr bool TAIL = NB > 0;
+    constexpr int SLOT_BYTES = TILE * D * 2;           // one K or one V tile
     constexpr int NBA = NB > 0 ? NB : 1;               // array extent (no zero-length arrays)
     pdl_enter();
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -183,7 +187,8 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
             const int pi = warp == 0 ? 0 : warp - 1;       // producer index 0..2
             TileCursor cur;
             cur.seek(p, start_b, start_prefix, t_begin, TILE);
-            const int page_in_tile = (lane >> 1) & 7, half = lane & 1;   // lane l < 16: page l/2, dims half l%2
+            // lane l < 16: page l/2, dims half l%2 (128 dims); lane l < 8: page l (64 dims, one half)
+            const int page_in_tile = D == 128 ? (lane >> 1) & 7 : lane & 7, half = D == 128 ? lane & 1 : 0;
             bool ok = true;
             long long tg = t_begin;
             for (uint32_t item = pi; ok && t_begin + (item >> 1) < t_end; item += 3) {
@@ -210,16 +215,15 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 if (!ok) break;
                 if (lane == 0) mbar_expect_tx(full, SLOT_BYTES);
                 __syncwarp();
-                if (lane < 16) {
-                    const uint32_t dst = smem_u32(ring + slot * SLOT_BYTES + half * (SLOT_BYTES / 2) +
-                                                  page_in_tile * 2048);
+                if (lane < D / 8) {
+                    const uint32_t dst = smem_u32(ring + slot * SLOT_BYTES + half * 16384 + page_in_tile * 2048);
                     tma_load_4d(dst, (item & 1) == 0 ? &k_map : &v_map, half * 64, 0, cur.g, phys, full);
                 }
             }
         } else if (t_end > t_begin && warp == 1) {
             // ================================================================ MMA issuer
             // the whole warp walks the schedule and waits; one elected lane issues
-            const uint32_t idesc_qk = instr_desc(false, TILE), idesc_pv = instr_desc(true, HD);
+            const uint32_t idesc_qk = instr_desc(false, TILE), idesc_pv = instr_desc(true, D);
             TileCursor cur;
             cur.seek(p, start_b, start_prefix, t_begin, TILE);
             uint32_t tile_no = 0;      // tiles of this block so far (ring position and S / P buffer parity)
@@ -241,8 +245,8 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     const uint32_t d = tmem + S_COL0 + (gu & 1) * TILE;
                     if (elect_one()) {
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks) {
-                            const uint32_t koff = ((ks >> 2) * (SLOT_BYTES / 2) + (ks & 3) * 32) >> 4;
+                        for (int ks = 0; ks < D / 16; ++ks) {
+                            const uint32_t koff = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
                             tc_mma_ts(d, tmem + Q_COL0 + ks * 8, kd + koff, idesc_qk, ks > 0);
                         }
                         tc_commit(smem_u32(&sh->s_full[gu & 1]));
@@ -260,7 +264,7 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     if (ok) ok = bounded_wait(smem_u32(&sh->full[slot]), (item / n_slots) & 1, abort_flag, p.device_status);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t vd = smem_desc(smem_u32(ring + slot * SLOT_BYTES), SLOT_BYTES / 2, 1024);
+                    const uint64_t vd = smem_desc(smem_u32(ring + slot * SLOT_BYTES), 16384, 1024);
                     const uint32_t pa = tmem + S_COL0 + (gu & 1) * TILE;      // P overlays S, TILE/2 columns
                     const uint32_t d = tmem + O_COL0;
                     if (elect_one()) {
@@ -309,9 +313,9 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 // this thread has seen the last S of that segment, and S follows all Q K^T in order.
                 if (warp_active) {
                     const uint4 *src = reinterpret_cast<const uint4 *>(
-                        static_cast<const __nv_bfloat16 *>(p.q) + q_row * HD);
+                        static_cast<const __nv_bfloat16 *>(p.q) + q_row * D);
 #pragma unroll
-                    for (int hf = 0; hf < 2; ++hf) {
+                    for (int hf = 0; hf < D / 64; ++hf) {
                         uint32_t qv[32];
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
@@ -376,7 +380,7 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                         tc_fence_after();
                         const float f = (rescale && ti > 0) ? factor : 1.f;
 #pragma unroll
-                        for (int ch = 0; ch < 4; ++ch) {
+                        for (int ch = 0; ch < D / 32; ++ch) {
                             uint32_t o[32];
                             tc_ld32(o_addr + ch * 32, o);
 #pragma unroll
@@ -427,9 +431,9 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     // padding rows: nothing to write
                 } else if (whole) {
                     const float inv = 1.f / l_sum;
-                    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.o) + q_row * HD;
+                    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.o) + q_row * D;
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
+                    for (int ch = 0; ch < D / 32; ++ch) {
                         uint32_t o[32];
                         tc_ld32(o_addr + ch * 32, o);
                         if (row_ok) {
@@ -449,9 +453,9 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                 } else {
                     // partial: fp32 O row, then max and sum; slot 0 = the block's first segment
                     float *slot = a.ws_part + ((size_t)blockIdx.x * 2 + (seg_no == 0 ? 0 : 1)) * part_slot_floats(a.slot_rows);
-                    float *orow = slot + (size_t)r * HD;
+                    float *orow = slot + (size_t)r * HD;          // 128-float pitch for both head sizes
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
+                    for (int ch = 0; ch < D / 32; ++ch) {
                         uint32_t o[32];
                         tc_ld32(o_addr + ch * 32, o);
                         if (row_ok) {
@@ -780,37 +784,39 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
 // ---------------------------------------------------------------------------- host side
 bool attn_tq_supported(const sv_attn_params &p)
 {
-    if (p.head_dim != HD || p.pool == nullptr || !p.pool->has_maps) return false;
+    if ((p.head_dim != 128 && p.head_dim != 64) || p.pool == nullptr || !p.pool->has_maps) return false;
     if (p.batch > MAX_BATCH_TC) return false;
     const int rows = (p.hq / p.hkv) * (p.gamma_max + 1);
-    return rows >= 1 && rows <= 128 + TAIL_ROWS;
+    return rows >= 1 && rows <= (p.head_dim == 128 ? 128 + TAIL_ROWS : 128);
 }
 
 int attn_tq_slot_rows(int rows) { return rows > 128 ? 128 + TAIL_ROWS : 128; }
 static int g_tail_blocks(int rows) { return rows <= 128 ? 0 : (rows - 128 + 7) / 8; }
 
-template <int NB>
+template <int NB, int D>
 static sv_status launch_tq(AttnTcLaunch &a, const sv_attn_params &p, int grid, cudaStream_t stream)
 {
     constexpr bool TAIL = NB > 0;
+    constexpr int slot_bytes = TILE * D * 2;
     const size_t budget = 227 * 1024;
     const size_t fixed = (TAIL ? sizeof(TailMerge) : 0) + ((sizeof(Shared) + 127) & ~(size_t)127);
-    a.n_slots = (int)((budget - fixed) / SLOT_BYTES);
+    a.n_slots = (int)((budget - fixed) / slot_bytes);
     if (a.n_slots > 8) a.n_slots = 8;
     if (a.n_slots < 4) return SV_EUNSUPPORTED;
-    const size_t smem = fixed + (size_t)a.n_slots * SLOT_BYTES;
-    if (cudaFuncSetAttribute(attn_tq_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+    const size_t smem = fixed + (size_t)a.n_slots * slot_bytes;
+    if (cudaFuncSetAttribute(attn_tq_kernel<NB, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
         return SV_ECUDA;
-    return launch_kernel(false, attn_tq_kernel<NB>, grid, TAIL ? 384 : 256, smem, stream, a, p.pool->k_map, p.pool->v_map);
+    return launch_kernel(false, attn_tq_kernel<NB, D>, grid, TAIL ? 384 : 256, smem, stream, a, p.pool->k_map, p.pool->v_map);
 }
 
 sv_status launch_attn_tq_main(AttnTcLaunch &a, const sv_attn_params &p, int grid, cudaStream_t stream)
 {
+    if (p.head_dim == 64) return launch_tq<0, 64>(a, p, grid, stream);
     switch (g_tail_blocks(a.group * (p.gamma_max + 1))) {
-        case 0: return launch_tq<0>(a, p, grid, stream);
-        case 1: return launch_tq<1>(a, p, grid, stream);
-        default: return launch_tq<2>(a, p, grid, stream);
+        case 0: return launch_tq<0, 128>(a, p, grid, stream);
+        case 1: return launch_tq<1, 128>(a, p, grid, stream);
+        default: return launch_tq<2, 128>(a, p, grid, stream);
     }
 }
 

@@ -250,6 +250,18 @@ def test_bf16_logits_small_and_odd_vocabularies(V):
     check_accept(bf16_rounded(li), cfg.temperature, g, cu_q, cu_d, cfg.gamma_max, bf16=True)
 
 
+@pytest.mark.parametrize("T", [0.05, 0.2, 4.0])
+def test_low_and_high_temperatures_keep_the_ratio_bound(T):
+    """The device forms ln Z from float32 exponentials of x * log2(e)/T - ref.  At a small temperature the products
+    are large (|x| / T up to ~200 here) and the reference nearly cancels them: the split of log2(e)/T into two
+    floats and the fused multiply-adds must keep the ratio within 1e-6 of the float64 one (check_accept asserts
+    it for every evaluated position), or decisions outside the flagged window would flip."""
+    cfg = synth.VerifyConfig("temp", 12, 1, 1, 64, 32000, 32, 32, 1, 6, 6, T, 0.6, seed=1000 + int(T * 100))
+    li, g, cu_q, cu_d = case(cfg)
+    gpu, ref, n_pos, n_tok = check_accept(li, T, g, cu_q, cu_d, cfg.gamma_max)
+    assert np.isfinite(ref.ratio).sum() >= 12
+
+
 def test_greedy_rows_without_an_argmax_set_the_status_bit():
     """T = 0: a target row that is all -inf, or holds a NaN or +inf, has no argmax.  The header promises
     SV_DEV_NONFINITE, no accepted drafts and -1 tokens for such a sequence, and nothing else changes."""
