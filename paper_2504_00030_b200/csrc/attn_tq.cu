@@ -22,6 +22,7 @@
 // hand-offs are mbarriers; every wait is bounded, an expired wait sets SV_DEV_TIMEOUT and
 // drains the block.
 #include "attn_sched.cuh"
+#include "attn_softmax.cuh"
 #include "tc_ptx.cuh"
 
 #include <math_constants.h>
@@ -37,7 +38,6 @@ constexpr int Q_COL0 = 384;                        // the query rows (bf16 pairs
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int TAIL_ROWS = 16;
 constexpr int SEG_COST = 6;                        // starting a pair costs about as much as six tiles (fitted: 5.8 us per pair against 1.5 us per tile; 3, 4 and 8 measured slower)
-constexpr float RESCALE_THRESHOLD = 8.f;           // log2 units: P <= 2^8 before a lazy rescale
 
 struct Shared {
     uint64_t full[8];        // ring slot filled by TMA
@@ -90,11 +90,6 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x)
     uint32_t y;
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
     return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t *>(&h);
 }
 
 }  // namespace tq
@@ -341,78 +336,12 @@ attn_tq_kernel(const AttnTcLaunch a, const __grid_constant__ CUtensorMap k_map,
                     tc_fence_after();
                     const int tok0 = (cur.t + ti) * TILE;
                     const bool need_mask = tok0 + TILE - 1 > L - R;    // some row cannot see the whole tile
-                    uint32_t s[TILE];
-#pragma unroll
-                    for (int ch = 0; ch < TILE / 32; ++ch) tc_ld32_nowait(s_addr + ch * 32, s + ch * 32);
-                    tc_wait_ld();
-                    if (need_mask) {
-#pragma unroll
-                        for (int c = 0; c < TILE; ++c)
-                            if (tok0 + c > pos) s[c] = 0xff800000u;     // -inf
-                    }
-                    float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
-#pragma unroll
-                    for (int c = 0; c < TILE; c += 4) {
-                        m0 = fmaxf(m0, __uint_as_float(s[c]));
-                        m1 = fmaxf(m1, __uint_as_float(s[c + 1]));
-                        m2 = fmaxf(m2, __uint_as_float(s[c + 2]));
-                        m3 = fmaxf(m3, __uint_as_float(s[c + 3]));
-                    }
-                    const float m_tile = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * c_scale;
-                    float factor = 1.f;
-                    bool rescale = false;
-                    if (m_tile > m_ref + RESCALE_THRESHOLD || m_ref == -CUDART_INF_F) {
-                        if (m_tile > -CUDART_INF_F) {
-                            rescale = (m_ref > -CUDART_INF_F);
-                            factor = rescale ? ex2_approx(m_ref - m_tile) : 1.f;
-                            m_ref = m_tile;
-                        }
-                    }
-                    const float m_use = (m_ref == -CUDART_INF_F) ? 0.f : m_ref;
-                    if (rescale) l_sum *= factor;
-                    // tensor-memory accesses are warp-wide: if any row of the warp has to rescale
-                    // its accumulator, the whole warp goes through (factor 1 elsewhere)
-                    if (__any_sync(0xffffffffu, rescale && ti > 0)) {
-                        // the accumulator may only be touched once the previous PV is complete
-                        ok = bounded_wait(smem_u32(&sh->o_done[(gu - 1) & 1]), ((gu - 1) >> 1) & 1, abort_flag,
-                                          p.device_status);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const float f = (rescale && ti > 0) ? factor : 1.f;
-#pragma unroll
-                        for (int ch = 0; ch < D / 32; ++ch) {
-                            uint32_t o[32];
-                            tc_ld32(o_addr + ch * 32, o);
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
-                            tc_st32(o_addr + ch * 32, o);
-                        }
-                    }
-                    // P = 2^(s*c - m_ref) as bf16 pairs, written over S (masked scores are -inf -> 0)
-                    float tile_sum = 0.f;
-#pragma unroll
-                    for (int ch = 0; ch < TILE / 32; ++ch) {
-                        float sum0 = 0.f, sum1 = 0.f;
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int c = 0; c < 32; c += 2) {
-                            const float e0 = ex2_approx(fmaf(__uint_as_float(s[ch * 32 + c]), c_scale, -m_use));
-                            const float e1 = ex2_approx(fmaf(__uint_as_float(s[ch * 32 + c + 1]), c_scale, -m_use));
-                            sum0 += e0;
-                            sum1 += e1;
-                            pk[c >> 1] = pack_bf16(e0, e1);
-                        }
-                        tile_sum += sum0 + sum1;
-                        asm volatile(
-                            "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-                            "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(
-                                s_addr + ch * 16),
-                            "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]),
-                            "r"(pk[7]), "r"(pk[8]), "r"(pk[9]), "r"(pk[10]), "r"(pk[11]), "r"(pk[12]),
-                            "r"(pk[13]), "r"(pk[14]), "r"(pk[15])
-                            : "memory");
-                    }
-                    l_sum += tile_sum;
+                    // the accumulator may only be rescaled once the previous PV is complete
+                    ok = softmax_tile<TILE, D / 32>(s_addr, o_addr, tok0, pos, need_mask, c_scale, ti == 0, m_ref, l_sum, [&]() {
+                        return bounded_wait(smem_u32(&sh->o_done[(gu - 1) & 1]), ((gu - 1) >> 1) & 1, abort_flag,
+                                            p.device_status);
+                    });
+                    if (!ok) break;
                     tc_wait_st();
                     tc_fence_before();
                     mbar_arrive(smem_u32(&sh->p_full[gu & 1]));
