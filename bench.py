@@ -201,7 +201,8 @@ def profiled_traffic_ratio():
         return None
 
 
-ATTN_KERNEL_SOURCES = ("attn_tq.cu", "attn_tc.cu", "attn_sched.cuh", "attn_common.cuh", "tc_ptx.cuh", "common.cuh")
+ATTN_KERNEL_SOURCES = ("attn_tq.cu", "attn_tc.cu", "attn_softmax.cuh", "attn_sched.cuh", "attn_common.cuh", "tc_ptx.cuh",
+                       "common.cuh")
 
 
 class VerifyStep:

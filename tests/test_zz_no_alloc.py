@@ -5,7 +5,7 @@ handed out completely at start-up, or a host framework that forbids (or would st
 cudaMalloc at the point of the call.  For them the library carries a fixed scratch array of its
 own.  This test calls that entry point through the C ABI, twice in a row on different inputs
 (the second call finds the first call's leftovers in the shared array), and checks every output
-against the regular entry point, which is itself checked against the oracle elsewhere.
+against the regular entry point; the counts and tokens are compared with the oracle as well.
 """
 import ctypes as C
 
@@ -53,6 +53,11 @@ def run_both(cfg, step):
     st = sv.load().spec_accept_sample_static(C.byref(p), C.c_void_p(torch.cuda.current_stream().cuda_stream))
     assert st == sv.SV_OK, sv.status_str(st)
     torch.cuda.synchronize()
+    # and against the oracle directly (counts and token ids, near ties followed as in the other accept tests)
+    from tests.harness import AcceptOut, compare_accept
+    out = AcceptOut(got["n"].cpu().numpy(), got["tok"].cpu().numpy(), got["ratio"].cpu().numpy(),
+                    got["lzp"].cpu().numpy(), got["lzq"].cpu().numpy(), 0, 0)
+    compare_accept(out, li, cfg.temperature, gamma, cu_q, cu_d, gmax)
     return ref, got
 
 
