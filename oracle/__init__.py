@@ -239,6 +239,28 @@ def draft_stop(draft_logits, temperature, tau, gamma, cu_d, tol=DRAFT_STOP_TOL):
     return n, top[:n_d], flag[:n_d]
 
 
+def draft_step(draft_logits, temperature, tau, u, gamma, cu_d, n_drafted, active, draft_tokens, top_prob,
+               tol=SAMPLE_TOL, conf_tol=DRAFT_STOP_TOL):
+    """One drafting step with the confidence stop (Section 4.2).  n_drafted, active (int32 [B]), draft_tokens
+    (int32 [n_d_rows]) and top_prob (float64 [n_d_rows]) are updated in place; returns (alt_token, sample_flag,
+    conf_flag), each [B]."""
+    lib = _load()
+    dl = _c(draft_logits, np.float32)
+    g, cd = _c(gamma, np.int32), _c(cu_d, np.int32)
+    B = len(g)
+    T = np.broadcast_to(np.asarray(temperature, np.float32), (B,)).copy()
+    uu = _c(u, np.float32)
+    for a, dt in ((n_drafted, np.int32), (active, np.int32), (draft_tokens, np.int32), (top_prob, np.float64)):
+        assert a.dtype == dt and a.flags.c_contiguous
+    alt = np.full(B, -1, np.int32)
+    sflag = np.zeros(B, np.uint8)
+    cflag = np.zeros(B, np.uint8)
+    lib.oracle_draft_step(_p(dl), ctypes.c_int64(dl.shape[1]), ctypes.c_int(dl.shape[1]), _p(T), ctypes.c_double(tau),
+                          _p(uu), _p(g), _p(cd), ctypes.c_int(B), ctypes.c_double(tol), ctypes.c_double(conf_tol),
+                          _p(n_drafted), _p(active), _p(draft_tokens), _p(top_prob), _p(alt), _p(sflag), _p(cflag))
+    return alt, sflag, cflag
+
+
 def cost_model(n_tokens, alpha, gamma, c):
     """Inference cost of Eq. 2-6 in units of T_draft."""
     return float(_load().oracle_cost_model(n_tokens, alpha, gamma, c))

@@ -429,6 +429,60 @@ void oracle_draft_stop(const float *draft_logits, int64_t row_stride, int vocab,
     }
 }
 
+/*
+ * One drafting step with the confidence stop (paper Section 4.2: the draft model's top
+ * probability is looked at while it drafts, and drafting ends once it falls below tau).
+ *
+ * Row b of draft_logits holds sequence b's draft logits for its next position.  For every
+ * sequence with active[b] != 0 (and n_drafted[b] < gamma[b]):
+ *     q = softmax(d / T);  token ~ q by inverse CDF with u[b]  (T == 0: token = argmax d, lowest index)
+ *     c = max_k q_k                                                (T == 0: c = 1)
+ *     draft_tokens[cu_d[b] + n_drafted[b]] = token, top_prob[same] = c, n_drafted[b] += 1
+ *     active[b] = (c >= tau) && (n_drafted[b] < gamma[b])
+ * The token drawn at a position whose confidence is below tau is kept (it is the last one
+ * drafted), as in oracle_draft_stop.  Sequences that are not active are left untouched.
+ * alt_token / sample_flag report a draw within tol of a CDF edge (see inv_cdf); conf_flag[b] = 1
+ * when |c - tau| < conf_tol (either decision is legal there).
+ */
+void oracle_draft_step(const float *draft_logits, int64_t row_stride, int vocab, const float *temperature,
+                       double tau, const float *u, const int32_t *gamma, const int32_t *cu_d, int batch,
+                       double tol, double conf_tol, int32_t *n_drafted, int32_t *active,
+                       int32_t *draft_tokens, double *top_prob, int32_t *alt_token, uint8_t *sample_flag,
+                       uint8_t *conf_flag)
+{
+    double *q = (double *)malloc((size_t)(vocab > 0 ? vocab : 1) * sizeof(double));
+    for (int b = 0; b < batch; ++b) {
+        alt_token[b] = -1;
+        sample_flag[b] = 0;
+        conf_flag[b] = 0;
+        if (!active[b]) continue;
+        if (n_drafted[b] >= gamma[b]) { active[b] = 0; continue; }
+        const float *d = draft_logits + (int64_t)b * row_stride;
+        const double T = (double)temperature[b];
+        int token;
+        double c = 1.0;
+        if (T > 0.0) {
+            softmax_f64(d, vocab, T, q);
+            int alt; uint8_t fl;
+            token = inv_cdf(q, vocab, (double)u[b], tol, &alt, &fl);
+            alt_token[b] = alt;
+            sample_flag[b] = fl;
+            c = 0.0;
+            for (int k = 0; k < vocab; ++k)
+                if (q[k] > c) c = q[k];
+        } else {
+            token = argmax_lowest(d, vocab);
+        }
+        const int pos = cu_d[b] + n_drafted[b];
+        draft_tokens[pos] = token;
+        top_prob[pos] = c;
+        conf_flag[b] = fabs(c - tau) < conf_tol ? 1 : 0;
+        n_drafted[b] += 1;
+        active[b] = (c >= tau) && (n_drafted[b] < gamma[b]);
+    }
+    free(q);
+}
+
 /* gamma = gamma0, gbar = gamma0 for every sequence, plus the prefix sums. */
 void oracle_gamma_tune_init(double *gamma_bar, int32_t *gamma, int32_t *cu_q, int32_t *cu_d,
                             int batch, int gamma0, int gamma_max, int padded_rows)
