@@ -371,6 +371,55 @@ size_t spec_draft_stop_workspace_bytes(int32_t batch, int32_t gamma_max, int32_t
 sv_status spec_draft_stop(const sv_draft_stop_params *p, void *workspace_device, size_t workspace_bytes,
                           void *stream);
 
+/* ---------------------------------------------------------------- GammaTune+ drafting step */
+/*
+ * Paper Section 4.2, the draft side: one drafting step of every sequence that
+ * is still drafting.  Row b of draft_logits holds sequence b's draft logits for
+ * its next position.  For every b with active[b] != 0 and n_drafted[b] < gamma[b]:
+ *     q = softmax(d_b / T);  token ~ q by inverse CDF in vocabulary order with
+ *     u_sample[b] (the smallest k with sum_{j<=k} q_j > u * sum_j q_j;
+ *     T == 0: token = argmax, lowest index on ties);  c = max_k q_k (T == 0: 1)
+ *     draft_tokens[cu_d[b] + n_drafted[b]] = token, top_prob[same] = c,
+ *     n_drafted[b] += 1,  active[b] = (c >= tau) && (n_drafted[b] < gamma[b]).
+ * The token drawn at a position whose confidence is below tau is kept, as in
+ * spec_draft_stop; a loop of these steps from n_drafted = 0 and active = 1 ends
+ * with the n_drafted that spec_draft_stop gives for the same rows, and with the
+ * tokens where spec_accept_sample reads them.  Sequences that are not active are
+ * not read and not written; one with n_drafted[b] >= gamma[b] only has active[b]
+ * cleared.  A row whose softmax sum is not finite (NaN or +inf logits) sets
+ * SV_DEV_NONFINITE, stores token -1 and clears active[b].
+ * Arithmetic: the top probability from float32 exponentials summed in float64
+ * (as spec_draft_stop), evaluated and compared with tau in float64; the token
+ * from a float64 pass over the row (as the bonus token of spec_accept_sample).
+ */
+typedef struct sv_draft_step_params {
+    const float *draft_logits;    /* device fp32 [batch, row_stride] (bf16 values if logits_bf16) */
+    int64_t row_stride;           /* elements between rows (>= vocab) */
+    int32_t vocab;
+    float temperature;            /* used when temperature_per_seq is NULL */
+    const float *temperature_per_seq; /* device [batch] or NULL */
+    float tau;                    /* threshold in [0, 1] */
+    const float *u_sample;        /* device [batch], in [0,1); may be NULL if every temperature is 0 */
+    const int32_t *gamma;         /* device [batch]: draft lengths issued by the controller */
+    const int32_t *cu_d;          /* device [batch+1]: first draft row of each sequence */
+    int32_t batch;
+    int32_t gamma_max;            /* bound on gamma[b] */
+    int32_t *n_drafted;           /* device in/out [batch] */
+    int32_t *active;              /* device in/out [batch] */
+    int32_t *draft_tokens;        /* device out [n_d_rows] */
+    double *top_prob;             /* device out [n_d_rows] or NULL */
+    uint32_t *device_status;      /* device, one word or NULL */
+    int32_t logits_bf16;          /* as in sv_accept_params */
+} sv_draft_step_params;
+
+size_t spec_draft_step_workspace_bytes(int32_t batch, int32_t vocab);
+
+/* Four launches on `stream`; nothing is read back.  Errors before any launch: SV_EINVAL (null pointers,
+ * sizes <= 0, row_stride < vocab, tau outside [0, 1], u_sample NULL with a positive temperature),
+ * SV_EWORKSPACE, SV_EALIGN (workspace not 16-byte aligned). */
+sv_status spec_draft_step(const sv_draft_step_params *p, void *workspace_device, size_t workspace_bytes,
+                          void *stream);
+
 /* ---------------------------------------------------------------- whole step from host buffers */
 /*
  * One verify step whose per-step inputs start in HOST memory: copies q,

@@ -26,7 +26,7 @@ EXPORTS = (
     "spec_verify_attn_workspace_bytes", "spec_verify_attn", "spec_accept_sample_workspace_bytes",
     "spec_accept_sample", "spec_accept_sample_static", "gamma_tune_update", "gamma_tune_init",
     "spec_verify_step_host", "spec_draft_stop_workspace_bytes", "spec_draft_stop", "spec_kv_append",
-    "sv_selftest_wait_expiry", "spec_verify_attn_layers",
+    "sv_selftest_wait_expiry", "spec_verify_attn_layers", "spec_draft_step_workspace_bytes", "spec_draft_step",
 )
 
 
@@ -90,6 +90,15 @@ class DraftStopParams(C.Structure):
                 ("logits_bf16", C.c_int32)]
 
 
+class DraftStepParams(C.Structure):
+    _fields_ = [("draft_logits", C.c_void_p), ("row_stride", C.c_int64), ("vocab", C.c_int32),
+                ("temperature", C.c_float), ("temperature_per_seq", C.c_void_p), ("tau", C.c_float),
+                ("u_sample", C.c_void_p), ("gamma", C.c_void_p), ("cu_d", C.c_void_p), ("batch", C.c_int32),
+                ("gamma_max", C.c_int32), ("n_drafted", C.c_void_p), ("active", C.c_void_p),
+                ("draft_tokens", C.c_void_p), ("top_prob", C.c_void_p), ("device_status", C.c_void_p),
+                ("logits_bf16", C.c_int32)]
+
+
 class StepHostIO(C.Structure):
     _fields_ = [("q_host", C.c_void_p), ("target_logits_host", C.c_void_p),
                 ("draft_logits_host", C.c_void_p), ("draft_tokens_host", C.c_void_p),
@@ -141,6 +150,10 @@ def load():
         lib.spec_draft_stop_workspace_bytes.argtypes = [C.c_int32] * 3
         lib.spec_draft_stop.restype = C.c_int32
         lib.spec_draft_stop.argtypes = [C.POINTER(DraftStopParams), C.c_void_p, C.c_size_t, C.c_void_p]
+        lib.spec_draft_step_workspace_bytes.restype = C.c_size_t
+        lib.spec_draft_step_workspace_bytes.argtypes = [C.c_int32] * 2
+        lib.spec_draft_step.restype = C.c_int32
+        lib.spec_draft_step.argtypes = [C.POINTER(DraftStepParams), C.c_void_p, C.c_size_t, C.c_void_p]
         lib.spec_verify_step_host.restype = C.c_int32
         lib.spec_verify_step_host.argtypes = [C.POINTER(StepHostIO), C.POINTER(AttnParams), C.c_void_p,
                                               C.c_size_t, C.POINTER(AcceptParams), C.c_void_p,
@@ -440,6 +453,45 @@ def spec_draft_stop(draft_logits, temperature, tau, gamma, cu_d, gamma_max, n_dr
                           device_status, temperature_per_seq)
     _check("spec_draft_stop",
            load().spec_draft_stop(C.byref(p), workspace.data_ptr(), _nbytes(workspace), _stream(stream)))
+
+
+# --------------------------------------------------------------------------- GammaTune+ drafting step
+def spec_draft_step_workspace_bytes(batch, vocab) -> int:
+    return int(load().spec_draft_step_workspace_bytes(batch, vocab))
+
+
+def draft_step_params(draft_logits, temperature, tau, u_sample, gamma, cu_d, gamma_max, n_drafted, active,
+                      draft_tokens, top_prob=None, device_status=None, temperature_per_seq=None) -> DraftStepParams:
+    p = DraftStepParams()
+    ldt = draft_logits.dtype if draft_logits.dtype == torch.bfloat16 else torch.float32       # float32 or bf16 logits
+    p.logits_bf16 = int(ldt == torch.bfloat16)
+    p.draft_logits = _dev(draft_logits, ldt, "draft_logits")
+    p.row_stride = draft_logits.stride(0)
+    p.vocab = draft_logits.shape[-1]
+    p.temperature = float(temperature)
+    p.temperature_per_seq = _dev(temperature_per_seq, torch.float32, "temperature_per_seq", True)
+    p.tau = float(tau)
+    p.u_sample = _dev(u_sample, torch.float32, "u_sample", True)
+    p.gamma = _dev(gamma, torch.int32, "gamma")
+    p.cu_d = _dev(cu_d, torch.int32, "cu_d")
+    p.batch = gamma.shape[0]
+    p.gamma_max = gamma_max
+    p.n_drafted = _dev(n_drafted, torch.int32, "n_drafted")
+    p.active = _dev(active, torch.int32, "active")
+    p.draft_tokens = _dev(draft_tokens, torch.int32, "draft_tokens")
+    p.top_prob = _dev(top_prob, torch.float64, "top_prob", True)
+    p.device_status = _dev(device_status, torch.int32, "device_status", True)
+    return p
+
+
+def spec_draft_step(draft_logits, temperature, tau, u_sample, gamma, cu_d, gamma_max, n_drafted, active,
+                    draft_tokens, workspace, top_prob=None, device_status=None, temperature_per_seq=None,
+                    stream=None):
+    """One drafting step with the confidence stop (asynchronous): token, top probability, n_drafted, active."""
+    p = draft_step_params(draft_logits, temperature, tau, u_sample, gamma, cu_d, gamma_max, n_drafted, active,
+                          draft_tokens, top_prob, device_status, temperature_per_seq)
+    _check("spec_draft_step",
+           load().spec_draft_step(C.byref(p), workspace.data_ptr(), _nbytes(workspace), _stream(stream)))
 
 
 def gamma_tune_init(gamma_bar, gamma, cu_q, cu_d, config: GammaConfig, gamma0: int, stream=None):

@@ -25,6 +25,8 @@
 #include "common.cuh"
 #include "row_stream.cuh"
 
+#include "row_sample.cuh"
+
 #include <math_constants.h>
 
 namespace sv {
@@ -47,13 +49,6 @@ struct __align__(16) RowPartial {
     int32_t bad;    // greedy rows: nonzero if the slice held a NaN (or +inf beside -inf)
 };
 
-// what the decision leaves for the sampling pass
-struct SeqRecord {
-    double sum_p_hat, sum_q_hat;  // first-pass sums of the sampled rows (at ref_p / ref_q)
-    float ref_p, ref_q;
-    int32_t n;                    // first rejection (gamma if none)
-    int32_t mode;                 // 0: nothing to sample (greedy or failed), 1: residual, 2: bonus row
-};
 
 struct AcceptLaunch {
     sv_accept_params p;
@@ -67,6 +62,7 @@ struct AcceptLaunch {
     int n_seg;
     int splits;
     int vec_ok;             // 128-bit loads legal for every row
+    int row_per_seq;        // the sampling pass alone, on row b of target_logits for sequence b, token to out_tokens[b]
 };
 
 // shared scratch of the decision
@@ -484,7 +480,7 @@ __device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const Seq
     const bool residual = rec.mode == 1;
     const int V = p.vocab, n_seg = a.n_seg, n = rec.n;
     const double c = 1.4426950408889634 / (double)seq_temperature(p, b);
-    const void *trow = logit_row<BF16>(p.target_logits, p.cu_q[b] + n, p.row_stride);
+    const void *trow = logit_row<BF16>(p.target_logits, a.row_per_seq ? b : p.cu_q[b] + n, p.row_stride);
     const void *drow = residual ? logit_row<BF16>(p.draft_logits, p.cu_d[b] + n, p.row_stride) : nullptr;
     const bool vec = a.vec_ok != 0;
     const double ref_p = (double)rec.ref_p, ref_q = (double)rec.ref_q;
@@ -615,7 +611,7 @@ __device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const Seq
         }
         y = last_pos;
     }
-    if (lane == 0) p.out_tokens[(long long)b * (p.gamma_max + 1) + n] = y;
+    if (lane == 0) p.out_tokens[a.row_per_seq ? (long long)b : (long long)b * (p.gamma_max + 1) + n] = y;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -646,7 +642,7 @@ accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
     const bool residual = rec.mode == 1;
     const int V = p.vocab, n_seg = a.n_seg;
     const double c = 1.4426950408889634 / (double)seq_temperature(p, b);
-    const void *trow = logit_row<BF16>(p.target_logits, p.cu_q[b] + rec.n, p.row_stride);
+    const void *trow = logit_row<BF16>(p.target_logits, a.row_per_seq ? b : p.cu_q[b] + rec.n, p.row_stride);
     const void *drow = residual ? logit_row<BF16>(p.draft_logits, p.cu_d[b] + rec.n, p.row_stride) : nullptr;
     const bool vec = a.vec_ok != 0;
     const double ref_p = (double)rec.ref_p, ref_q = (double)rec.ref_q;
@@ -825,6 +821,7 @@ static sv_status launch_accept(const sv_accept_params *p, void *scratch, int sli
     if (splits > (a.n_seg + 7) / 8) splits = (a.n_seg + 7) / 8;
     if (splits < 1 || !any_sampling) splits = 1;
     a.splits = splits;
+    a.row_per_seq = 0;
 
     const long long n_items = (long long)p->batch * (2 * p->gamma_max + 1) * a.n_slices;
     const long long blocks_needed = (n_items + RS_THREADS / 32 - 1) / (RS_THREADS / 32);
@@ -841,6 +838,51 @@ static sv_status launch_accept(const sv_accept_params *p, void *scratch, int sli
     const long long cap = (long long)blocks_per_sm_of[dev][bf16] * sm_count();
     const int rs_grid = (int)(blocks_needed < cap ? blocks_needed : cap);
     return bf16 ? launch_kernels<true>(a, rs_grid, stream) : launch_kernels<false>(a, rs_grid, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// The sampling pass alone (row_sample.cuh): one row per sequence, records prepared by the caller's kernel.
+// ---------------------------------------------------------------------------------------------
+static int row_sample_splits(int batch, int n_seg)
+{
+    int splits = (2 * 4 * sm_count()) / batch;
+    if (splits > MAX_SPLITS) splits = MAX_SPLITS;
+    if (splits > (n_seg + 7) / 8) splits = (n_seg + 7) / 8;
+    return splits < 1 ? 1 : splits;
+}
+
+size_t row_sample_scratch_bytes(int batch, int vocab)
+{
+    const size_t n_seg = ((size_t)vocab + SEG - 1) / SEG;
+    return align256((size_t)batch * 3 * n_seg * sizeof(double)) + align256((size_t)batch * MAX_SPLITS * 2 * sizeof(double));
+}
+
+sv_status launch_row_sample(const RowSampleArgs &r, cudaStream_t stream)
+{
+    AcceptLaunch a;
+    memset(&a, 0, sizeof(a));
+    a.p.target_logits = static_cast<const float *>(r.logits);
+    a.p.logits_bf16 = r.logits_bf16;
+    a.p.row_stride = r.row_stride;
+    a.p.vocab = r.vocab;
+    a.p.batch = r.batch;
+    a.p.temperature = r.temperature;
+    a.p.temperature_per_seq = r.temperature_per_seq;
+    a.p.u_sample = r.u_sample;
+    a.p.out_tokens = r.out_tokens;
+    a.p.device_status = r.device_status;
+    a.records = const_cast<SeqRecord *>(r.records);
+    a.done = r.done;
+    a.n_seg = (r.vocab + SEG - 1) / SEG;
+    a.seg = static_cast<double *>(r.scratch);
+    a.totals = reinterpret_cast<double *>(static_cast<uint8_t *>(r.scratch) +
+                                          align256((size_t)r.batch * 3 * a.n_seg * sizeof(double)));
+    a.splits = row_sample_splits(r.batch, a.n_seg);
+    a.vec_ok = logits_vec_ok(r.logits, r.row_stride, r.logits_bf16 != 0);
+    a.row_per_seq = 1;
+    const unsigned grid = (unsigned)(a.splits * r.batch);
+    return r.logits_bf16 ? launch_kernel(true, accept_sample_kernel<true>, grid, SEG_THREADS, 0, stream, a)
+                         : launch_kernel(true, accept_sample_kernel<false>, grid, SEG_THREADS, 0, stream, a);
 }
 
 }  // namespace sv
