@@ -468,6 +468,22 @@ def run_ours(args):
     t_ds = median_us(lambda: check(lib.spec_draft_stop(C.byref(dp), ws_d.data_ptr(), ws_d.numel(), sptr), "draft_stop"))
     ds_bytes = int(gamma.sum()) * cfg.vocab * 4
 
+    # ---- one drafting step with the confidence stop (not part of the step above): a row of draft logits per
+    # sequence (the first B rows of the block's draft logits), token and top probability, state advanced
+    n_st = torch.zeros(B, dtype=torch.int32, device=DEV)
+    act_st = torch.ones(B, dtype=torch.int32, device=DEV)
+    tok_st = torch.zeros(max(int(cu_d[-1]), 1), dtype=torch.int32, device=DEV)
+    ws_st = torch.empty(max(256, sv.spec_draft_step_workspace_bytes(B, cfg.vocab)), dtype=torch.uint8, device=DEV)
+    stp = sv.draft_step_params(vs.dl[:B], cfg.temperature, 0.0, vs.us, vs.g, vs.cd, gmax, n_st, act_st, tok_st,
+                               device_status=status)
+
+    def draft_step_once():
+        n_st.zero_()            # every call drafts position 0 of every sequence again
+        act_st.fill_(1)
+        check(lib.spec_draft_step(C.byref(stp), ws_st.data_ptr(), ws_st.numel(), sptr), "draft_step")
+    t_st = median_us(draft_step_once)
+    st_bytes = B * cfg.vocab * 4
+
     # ---- accept / resample with the logits stored as bf16 (not part of the step above): same call, half the bytes
     tl16, dl16 = vs.tl.to(torch.bfloat16), vs.dl.to(torch.bfloat16)
     n16 = torch.zeros(B, dtype=torch.int32, device=DEV)
@@ -570,6 +586,9 @@ def run_ours(args):
     if clocks is not None and clocks.get("sm_mhz"):
         # the GPUs of a pool differ in the clock they hold; time x clock compares kernels across them
         line["step_us_x_sm_ghz"] = 1e3 * ms_step * clocks["sm_mhz"] / 1e3
+    line["draft_step"] = {"what": "one drafting step with the confidence stop (a draft row per sequence: token, top "
+                                  "probability, state), outside the timed step; includes two small fills",
+                          "us": t_st, "bytes": st_bytes, "gbs": st_bytes / (t_st * 1e-6) / 1e9}
     line["accept_bf16_logits"] = {"what": "spec_accept_sample on the same logits stored as bf16, outside the timed step",
                                   "us": t_a16, "bytes": a16_bytes, "gbs": a16_bytes / (t_a16 * 1e-6) / 1e9,
                                   "frac_of_measured": a16_bytes / (t_a16 * 1e-6) / 1e9 / peak}
