@@ -190,6 +190,13 @@ def _dev(t, dtype, name, allow_none=False):
     return t.data_ptr()
 
 
+def _dev_rows(t, dtype, name):
+    """Device pointer of a 2-D CUDA tensor whose rows are contiguous; the rows may be strided."""
+    if t is None or not t.is_cuda or t.dtype != dtype or t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise ValueError(f"{name} must be a 2-D CUDA tensor of {dtype} with contiguous rows")
+    return t.data_ptr()
+
+
 def _host(t, dtype, name, allow_none=False):
     if t is None:
         if allow_none:
@@ -465,7 +472,7 @@ def draft_step_params(draft_logits, temperature, tau, u_sample, gamma, cu_d, gam
     p = DraftStepParams()
     ldt = draft_logits.dtype if draft_logits.dtype == torch.bfloat16 else torch.float32       # float32 or bf16 logits
     p.logits_bf16 = int(ldt == torch.bfloat16)
-    p.draft_logits = _dev(draft_logits, ldt, "draft_logits")
+    p.draft_logits = _dev_rows(draft_logits, ldt, "draft_logits")     # e.g. position i of every block
     p.row_stride = draft_logits.stride(0)
     p.vocab = draft_logits.shape[-1]
     p.temperature = float(temperature)

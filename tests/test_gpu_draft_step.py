@@ -251,3 +251,75 @@ def test_one_step_at_the_largest_size():
     n, act = loop.step(d, 1.0, float(np.median(top)), r.random(B).astype(np.float32))
     assert int(loop.status.item()) == 0
     assert 0 < int(act.sum()) < B and (n == 1).all()
+
+
+def test_drafting_loop_feeds_the_verify_step_without_a_host_round_trip():
+    """Three speculative steps of a small batch, all state on the device: the draft tokens of every block come
+    from a loop of spec_draft_step calls (strided views of the block's draft rows, no copy), spec_accept_sample
+    reads them where they were written with n_drafted as its draft lengths, and the controller is told both.
+    Nothing is read back until the end; the oracle then takes the same steps."""
+    import dataclasses
+    from tests.harness import AcceptOut, compare_accept
+    cfg = synth.scaled(synth.CONFIGS["c2"], batch=3, gamma_max=6, gamma_lo=6, gamma_hi=6)
+    B, gmax, V, T, tau, steps = cfg.batch, cfg.gamma_max, cfg.vocab, 1.0, 0.012, 3
+    gcfg = sv.GammaConfig(0.5, 2.0, 1, gmax, sv.SV_GT_PROPOSED, True)
+    cu_q, cu_d = synth.padded_offsets(B, gmax)
+    full = np.full(B, gmax, np.int32)
+    rng = np.random.default_rng(31)
+    inputs = [synth.make_logits(cfg, full, cu_q, cu_d, step=t, sigma_noise=0.7, temperature=T) for t in range(steps)]
+    u_draft = [rng.random((gmax, B)).astype(np.float32) for _ in range(steps)]
+
+    gbar = torch.zeros(B, dtype=torch.float64, device=DEV)
+    g = torch.zeros(B, dtype=torch.int32, device=DEV)
+    sl = dev(np.full(B, 500, np.int32))
+    d_cq = torch.zeros(B + 1, dtype=torch.int32, device=DEV)
+    d_cd = torch.zeros(B + 1, dtype=torch.int32, device=DEV)
+    sv.gamma_tune_init(gbar, g, d_cq, d_cd, gcfg, 4)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    n_dr = torch.zeros((steps, B), dtype=torch.int32, device=DEV)
+    act = torch.zeros(B, dtype=torch.int32, device=DEV)
+    x = torch.full((steps, B * gmax), -1, dtype=torch.int32, device=DEV)
+    n_acc = torch.zeros((steps, B), dtype=torch.int32, device=DEV)
+    toks = torch.zeros((steps, B, gmax + 1), dtype=torch.int32, device=DEV)
+    traj = torch.zeros((steps, B), dtype=torch.int32, device=DEV)
+    ws_p = workspace(sv.spec_draft_step_workspace_bytes(B, V))
+    ws_s = workspace(sv.spec_accept_sample_workspace_bytes(B, gmax, V))
+    d_in = [(dev(li.target_logits), dev(li.draft_logits), dev(li.u_accept), dev(li.u_sample)) for li in inputs]
+    d_u = [dev(u) for u in u_draft]
+    for t in range(steps):
+        tl, dl, ua, us = d_in[t]
+        act.fill_(1)
+        rows = dl.view(B, gmax, V)
+        for i in range(gmax):
+            sv.spec_draft_step(rows[:, i], T, tau, d_u[t][i], g, d_cd, gmax, n_dr[t], act, x[t], ws_p,
+                               device_status=status)
+        sv.spec_accept_sample(tl, dl, x[t], ua, us, T, n_dr[t], d_cq, d_cd, gmax, n_acc[t], toks[t], ws_s,
+                              device_status=status)
+        sv.gamma_tune_update(n_acc[t], gbar, g, sl, d_cq, d_cd, gcfg, trajectory=traj, step=t,
+                             device_status=status, n_drafted=n_dr[t])
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    n_dr, x, n_acc, toks, traj = (a.cpu().numpy() for a in (n_dr, x, n_acc, toks, traj))
+
+    o_gbar, o_g, _, _ = oracle.gamma_tune_init(B, 4, gmax, True)
+    o_sl = np.full(B, 500, np.int32)
+    stopped_early = 0
+    for t in range(steps):
+        li = inputs[t]
+        st = (np.zeros(B, np.int32), np.ones(B, np.int32), np.full(B * gmax, -1, np.int32), np.full(B * gmax, np.nan))
+        for i in range(gmax):
+            d = li.draft_logits.reshape(B, gmax, V)[:, i]
+            alt, sflag, cflag = oracle.draft_step(d, T, tau, u_draft[t][i], o_g, cu_d, *st)
+            assert not sflag.any() and not cflag.any()          # these seeds meet no near tie
+        np.testing.assert_array_equal(n_dr[t], st[0])
+        np.testing.assert_array_equal(x[t], st[2])
+        stopped_early += int((st[0] < o_g).sum())
+        gpu = AcceptOut(n_acc[t], toks[t], None, None, None, 0, 0)
+        compare_accept(gpu, dataclasses.replace(li, draft_tokens=st[2]), T, st[0], cu_q, cu_d, gmax)
+        o_gbar, o_g, o_sl, _, _ = oracle.gamma_tune_update(n_acc[t], o_gbar, o_g, o_sl, gcfg.eta, gcfg.delta,
+                                                           gcfg.gamma_min, gcfg.gamma_max, gcfg.mode, True,
+                                                           n_drafted=st[0])
+        np.testing.assert_array_equal(traj[t], o_g)
+    assert stopped_early > 0
+    np.testing.assert_array_equal(gbar.cpu().numpy().view(np.int64), o_gbar.view(np.int64))
+    np.testing.assert_array_equal(sl.cpu().numpy(), o_sl)
