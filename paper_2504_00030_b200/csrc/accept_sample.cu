@@ -33,7 +33,9 @@ namespace sv {
 
 constexpr int RS_THREADS = 256;   // rowstats block (8 independent warps)
 constexpr int RS_UNROLL = 6;      // float4 loads in flight per lane: 61 registers, 32 warps per SM (4, 8, 12, 16 measured slower)
-constexpr int SEG = 128;          // vocabulary elements per sampling segment (one warp, float4 per lane)
+constexpr int CHUNK = 128;        // vocabulary elements a warp takes at a time (float4 per lane)
+constexpr int SEG_SUB = 4;         // chunks per sampling segment: one reduction and one record per segment
+constexpr int SEG = CHUNK * SEG_SUB;
 constexpr int SEG_THREADS = 256;
 constexpr int MAX_SPLITS = 64;    // blocks per sequence in the sampling kernel (small batches: enough blocks to fill the GPU)
 constexpr int MIN_SLICE = 2048;
@@ -566,10 +568,11 @@ __device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const Seq
     // resolve inside the segment; if rounding pushed the target past it, walk on; if nothing
     // qualifies, take the last positive weight.
     int y = -1, last_pos = -1;
-    int s = best;
+    const int n_chunk = (V + CHUNK - 1) / CHUNK;
+    int s = best * SEG_SUB;                      // from here on in chunks of 128 tokens
     if (best >= n_seg) { s = 0; base = 0.0; }    // target at or beyond the total: walk everything
-    for (; s < n_seg && y < 0; ++s) {
-        const int k0 = s * SEG + 4 * lane;
+    for (; s < n_chunk && y < 0; ++s) {
+        const int k0 = s * CHUNK + 4 * lane;
         double w[4], loc = 0.0;
         weights4(k0, w);
 #pragma unroll
@@ -598,8 +601,8 @@ __device__ __forceinline__ void pick_seq(const AcceptLaunch &a, int b, const Seq
     }
     if (y < 0) {
         // target at or beyond the total mass: last token with positive weight
-        for (int s2 = n_seg - 1; s2 >= 0 && last_pos < 0; --s2) {
-            const int k0 = s2 * SEG + 4 * lane;
+        for (int s2 = n_chunk - 1; s2 >= 0 && last_pos < 0; --s2) {
+            const int k0 = s2 * CHUNK + 4 * lane;
             double w[4];
             weights4(k0, w);
             int lp = -1;
@@ -653,46 +656,41 @@ accept_sample_kernel(const __grid_constant__ AcceptLaunch a)
     const int per = (n_seg + a.splits - 1) / a.splits;
     const int s_begin = sp * per, s_end = min(n_seg, s_begin + per);
     double tot_a = 0.0, tot_b = 0.0;
-    constexpr int UN = 1;               // segments whose loads are issued together
     constexpr int NW = SEG_THREADS / 32;
-    for (int s0 = s_begin + warp; s0 < s_end; s0 += UN * NW) {
-        float xt[UN][4], xd[UN][4];
-#pragma unroll
-        for (int q = 0; q < UN; ++q) {
-            const int s = s0 + q * NW;
-            if (s < s_end) {
-                logit_load4<BF16>(trow, s * SEG + 4 * lane, V, vec, xt[q]);
-                if (residual) logit_load4<BF16>(drow, s * SEG + 4 * lane, V, vec, xd[q]);
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < UN; ++q) {
-            const int s = s0 + q * NW;
-            if (s >= s_end) break;
+    for (int s = s_begin + warp; s < s_end; s += NW) {
+        {
             double sa = 0.0, sap = 0.0, sbp = 0.0, sb = 0.0;
-            if (residual) {
-                // the eight exponentials of this lane (four tokens, two rows) as overlapping chains
-                double y[8], w[8];
+#pragma unroll 1
+            for (int sub = 0; sub < SEG_SUB; ++sub) {
+                const int k0 = s * SEG + sub * CHUNK + 4 * lane;
+                if (k0 - 4 * lane >= V) break;                   // past the vocabulary (last segment)
+                float xt[4], xd[4];
+                logit_load4<BF16>(trow, k0, V, vec, xt);
+                if (residual) {
+                    logit_load4<BF16>(drow, k0, V, vec, xd);
+                    // the eight exponentials of this lane (four tokens, two rows) as overlapping chains
+                    double y[8], w[8];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    y[u] = (double)xt[q][u] * c - ref_p;
-                    y[4 + u] = (double)xd[q][u] * c - ref_q;
+                    for (int u = 0; u < 4; ++u) {
+                        y[u] = (double)xt[u] * c - ref_p;
+                        y[4 + u] = (double)xd[u] * c - ref_q;
+                    }
+                    exp2_f64_n<8>(y, w, s_tab);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const double ak = w[u], bk = w[4 + u];
+                        sa += ak;
+                        sb += bk;
+                        if (ak * z_ratio > bk) { sap += ak; sbp += bk; }
+                    }
+                } else {
+                    double y[4], w[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) y[u] = (double)xt[u] * c - ref_p;
+                    exp2_f64_n<4>(y, w, s_tab);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) sa += w[u];
                 }
-                exp2_f64_n<8>(y, w, s_tab);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const double ak = w[u], bk = w[4 + u];
-                    sa += ak;
-                    sb += bk;
-                    if (ak * z_ratio > bk) { sap += ak; sbp += bk; }
-                }
-            } else {
-                double y[4], w[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) y[u] = (double)xt[q][u] * c - ref_p;
-                exp2_f64_n<4>(y, w, s_tab);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) sa += w[u];
             }
             tot_a += sa;
             tot_b += sb;
