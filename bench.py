@@ -292,6 +292,36 @@ class VerifyStep:
         for i, _ in enumerate(self.calls()):
             if ev is not None: ev[i + 1].record(self.stream)
 
+    def graph_us(self, steps):
+        """The step captured once into a CUDA graph and replayed `steps` times: microseconds per replay, or None
+        if the capture is refused.  What a caller gains on the launch-bound small workloads."""
+        torch, C = self.torch, self.C
+        keep = (self.stream, self.sptr)
+        side = torch.cuda.Stream()
+        self.stream, self.sptr = side, C.c_void_p(side.cuda_stream)
+        try:
+            torch.cuda.synchronize()
+            with torch.cuda.stream(side):
+                self.step()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                self.step()
+            torch.cuda.synchronize()
+            for _ in range(3):
+                graph.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(steps):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            return 1e3 * e0.elapsed_time(e1) / steps
+        except RuntimeError:
+            return None
+        finally:
+            self.stream, self.sptr = keep
+
     def evolve(self, n):
         """The controller runs n steps on its own acceptance counts (no reset); the timed steps then start from
         the state it reached: a GammaTune-driven mix of draft lengths instead of gamma_max everywhere."""
@@ -353,7 +383,8 @@ def config_lines(sv, torch, dev, steps, peak):
                      "gamma_update_us": 1e3 * r["gamma"], "bytes": attn_b + acc_b,
                      "frac_of_8tbs": (attn_b + acc_b) / (us * 1e-6) / 8e12,
                      "frac_of_measured": (attn_b + acc_b) / (us * 1e-6) / 1e9 / peak,
-                     "verified_tokens_per_s": r["tokens"] / (us * 1e-6)}
+                     "verified_tokens_per_s": r["tokens"] / (us * 1e-6),
+                     "graph_step_us": vs.graph_us(steps)}       # the same step as one CUDA graph launch
         del vs
         torch.cuda.empty_cache()
     return out
