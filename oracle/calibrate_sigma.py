@@ -12,7 +12,7 @@ noise sigma on a grid:
 
 Inputs are the seeded synthetic logits of the workload (draft ~ N(0, 2^2), target = draft + N(0, sigma^2),
 V = 32000).  Run:  python -m oracle.calibrate_sigma [--rows 256]
-The chosen values are recorded in the design doc and used by the multi-step tests.
+The chosen values are the C4_SIGMA table of tests/test_gpu_step.py, used by the multi-step tests.
 """
 from __future__ import annotations
 
