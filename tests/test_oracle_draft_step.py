@@ -143,3 +143,12 @@ def test_inactive_sequences_are_left_alone_and_flags_are_raised():
     assert st[2][0] == -1 and st[0][0] == 0 and np.isnan(st[3][0])
     assert cflag[1] == 1                    # top probability 1/4 against tau = 1/4
     assert st[2][1] == 2 and sflag[1] == 1 and alt[1] == 1       # u = 1/2 sits on the CDF edge between 1 and 2
+
+
+def test_confidence_equal_to_the_threshold_keeps_drafting():
+    # q = 1/4 each and tau = 1/4: the stop needs c < tau (as in the block form), so the sequence stays active
+    st = state(1, 2)
+    one_step(np.zeros((1, 4), np.float32), 1.0, 0.25, [0.1], np.array([2], np.int32), np.array([0, 2], np.int32), st)
+    assert st[1][0] == 1 and st[0][0] == 1
+    n_block, _, _ = oracle.draft_stop(np.zeros((2, 4), np.float32), 1.0, 0.25, [2], [0, 2])
+    assert n_block[0] == 2
