@@ -311,7 +311,7 @@ __device__ __forceinline__ RowPartial load_partial(const RowPartial *q)
 // by groups of lanes, one group per row, its lanes over the slices (a shuffle butterfly);
 // warp 0 then evaluates the positions in parallel and lane 0 walks to the first rejection.
 // ---------------------------------------------------------------------------------------------
-constexpr int DEC_THREADS = 128;
+constexpr int DEC_THREADS = 512;   // 16 warps: the rows of a sequence merged in one or two passes (128 threads: six at c3, +14 us)
 
 template <bool BF16>
 __device__ __forceinline__ void decide_seq(const AcceptLaunch &a, int b, DecideScratch *sc, int tid, SeqRecord *rec_out)

@@ -115,7 +115,7 @@ draft_conf_rowstats_kernel(const __grid_constant__ DraftStopLaunch a)
     }
 }
 
-constexpr int DSD_THREADS = 128;
+constexpr int DSD_THREADS = 512;     // 16 warps: all positions of a sequence in one or two passes
 
 __global__ void __launch_bounds__(DSD_THREADS)
 draft_stop_decide_kernel(const __grid_constant__ DraftStopLaunch a)
